@@ -1,0 +1,440 @@
+/*
+ * CPU oracle for block-scaled e4m3 fast matrix multiplication.
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is a plain, slow, obviously-correct
+ * restatement of what the paper's fused block-scaled fp8 regime computes.  It
+ * shares no code with the CUDA library and is never on the product path; only
+ * the tests, the smoke check and the CPU-baseline leg of the benchmark load it.
+ *
+ * What it follows (paper sections / equations):
+ *   - bilinear algorithm  c = sum_r <U_r,a><V_r,b> W_r with a, b, c the
+ *     row-vectorised 2x2 block matrices (order 11,12,21,22)        [Sec. 2.1]
+ *   - fused regime: raw operand blocks stay unquantized; the encoded
+ *     combinations x_r, y_r are formed first (fp32) and then quantized;
+ *     the decoder W_r carries each product into the output
+ *                                                [Sec. 2.2, Assumption 1; App. D.1]
+ *   - block quantizer: scale = amax / 448 kept in fp32, the scaled block is
+ *     cast to e4m3 with round-to-nearest-even, and rescaled; groups of
+ *     1 x blk along the contracted axis on BOTH sides; a minimum-scale clamp
+ *     engages below amax = 1e-12                                    [App. E.2]
+ *   - recursion: the encoders / decoder are applied level by level (Kronecker
+ *     power); only the leaf combinations are quantized              [Sec. 3, App. E]
+ *   - error metric: relative Frobenius error against an fp64 product [App. E.2]
+ *
+ * Readings taken where the paper is silent (each also listed in the design notes):
+ *   - the block is scaled by multiplying with inv = fl32(448/amax_c); the stored
+ *     scale is s = fl32(amax_c/448); amax_c = max(amax, 1e-12f)
+ *   - linear combinations are evaluated in fp32 in quadrant order 11,12,21,22,
+ *     zero coefficients skipped, first term a rounded multiply, later terms a
+ *     single-rounded fused multiply-add
+ *   - values beyond +-448 after scaling saturate to +-448 (codes 0x7E / 0xFE)
+ *   - second scale mode (hardware-native deviation, labelled as such everywhere):
+ *     the scale is rounded UP to a power of two (UE8M0), e = ceil(log2(amax_c/448))
+ *   - products and the decode are carried in fp64 on exactly dequantized operands
+ *
+ * Pins: see tests/test_oracle_*.py (exhaustive e4m3 tables and midpoints,
+ * library cast cross-check, homogeneity of the quantizer, identity-quantizer
+ * runs equal to A*B, the paper's printed error figures).
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+#define ORACLE_MAX_RANK 8
+#define SCALE_FP32 0
+#define SCALE_UE8M0 1
+#define SCALE_IDENTITY 2 /* no quantization at all: used only to pin the bilinear algebra */
+
+/* ------------------------------------------------------------------ e4m3 */
+
+static uint32_t f32_bits(float x) { uint32_t u; memcpy(&u, &x, 4); return u; }
+static float bits_f32(uint32_t u) { float x; memcpy(&x, &u, 4); return x; }
+
+/* OCP e4m3 ("fn"): 1 sign, 4 exponent (bias 7), 3 mantissa bits; no infinity;
+ * S.1111.111 is NaN; largest finite 448 = 0x7E; smallest normal 2^-6;
+ * subnormal quantum 2^-9.  Round to nearest, ties to even; saturating. */
+uint8_t oracle_e4m3_encode(float y)
+{
+    uint32_t u = f32_bits(y);
+    uint8_t sign = (uint8_t)((u >> 31) << 7);
+    uint32_t au = u & 0x7fffffffu;
+    if (au > 0x7f800000u) return 0x7F;             /* NaN */
+    float a = bits_f32(au);
+    if (a >= 448.0f) return (uint8_t)(sign | 0x7E); /* saturate (also covers inf) */
+    if (a < 0.015625f) {                           /* below 2^-6: subnormal grid, quantum 2^-9 */
+        /* a * 512 is exact in fp32 (power-of-two scaling, result < 8) */
+        float t = a * 512.0f;
+        uint32_t q = (uint32_t)t;                  /* floor */
+        float frac = t - (float)q;                 /* exact */
+        if (frac > 0.5f || (frac == 0.5f && (q & 1u))) q += 1u;
+        return (uint8_t)(sign | q);                /* q == 8 is exactly code 0x08 = 2^-6 */
+    }
+    int e = (int)(au >> 23) - 127;                 /* -6 .. 8 */
+    uint32_t man = au & 0x7fffffu;
+    uint32_t keep = man >> 20;                     /* top 3 mantissa bits */
+    uint32_t rest = man & 0xfffffu;                /* 20 dropped bits */
+    if (rest > 0x80000u || (rest == 0x80000u && (keep & 1u))) keep += 1u;
+    if (keep == 8u) { keep = 0u; e += 1; }
+    uint32_t code = ((uint32_t)(e + 7) << 3) | keep;
+    if (code > 0x7Eu) code = 0x7Eu;                /* rounded past 448 */
+    return (uint8_t)(sign | code);
+}
+
+double oracle_e4m3_decode(uint8_t c)
+{
+    int s = c >> 7, e = (c >> 3) & 15, m = c & 7;
+    double v;
+    if (e == 15 && m == 7) return NAN;
+    if (e == 0) v = ldexp((double)m, -9);
+    else v = ldexp(1.0 + (double)m / 8.0, e - 7);
+    return s ? -v : v;
+}
+
+void oracle_e4m3_encode_array(const float *y, int64_t n, uint8_t *out)
+{
+    for (int64_t i = 0; i < n; ++i) out[i] = oracle_e4m3_encode(y[i]);
+}
+
+void oracle_e4m3_decode_array(const uint8_t *c, int64_t n, double *out)
+{
+    for (int64_t i = 0; i < n; ++i) out[i] = oracle_e4m3_decode(c[i]);
+}
+
+/* ------------------------------------------------------- block quantizer */
+
+typedef struct {
+    int blk;          /* block length along the contracted axis */
+    int mode;         /* SCALE_FP32 | SCALE_UE8M0 | SCALE_IDENTITY */
+    float amax_floor; /* minimum-scale clamp, 1e-12 in the paper */
+} qparams_t;
+
+/* Quantize one block of `blk` values x[0], x[stride], ...  Writes the codes with
+ * the same stride and returns the scale as a double-exact fp32 value.
+ * For UE8M0 the biased exponent byte is also returned through *e8. */
+static float quant_block(const float *x, int64_t stride, int blk, const qparams_t *qp,
+                         uint8_t *codes, int64_t cstride, uint8_t *e8)
+{
+    float amax = 0.0f;
+    for (int i = 0; i < blk; ++i) {
+        float a = fabsf(x[i * stride]);
+        if (a > amax) amax = a;
+    }
+    float amax_c = amax > qp->amax_floor ? amax : qp->amax_floor;
+    if (qp->mode == SCALE_FP32) {
+        float s = amax_c / 448.0f;
+        float inv = 448.0f / amax_c;
+        for (int i = 0; i < blk; ++i) {
+            float y = x[i * stride] * inv;
+            codes[i * cstride] = oracle_e4m3_encode(y);
+        }
+        if (e8) *e8 = 0;
+        return s;
+    }
+    /* UE8M0: smallest power of two >= amax_c/448 */
+    float s0 = amax_c / 448.0f;
+    uint32_t u = f32_bits(s0);
+    int ex = (int)(u >> 23);            /* biased; 0 for subnormal s0 */
+    uint32_t man = u & 0x7fffffu;
+    int e;
+    if (ex == 0) {
+        /* subnormal s0 = man * 2^-149 (man > 0 because amax_c > 0) */
+        int hi = 31 - __builtin_clz(man);
+        e = hi - 149 + ((man & (man - 1u)) ? 1 : 0);
+    } else {
+        e = ex - 127 + (man ? 1 : 0);
+    }
+    if (e < -127) e = -127;
+    if (e > 127) e = 127;
+    float inv = ldexpf(1.0f, -e);       /* exact, representable (possibly subnormal) */
+    for (int i = 0; i < blk; ++i) {
+        float y = x[i * stride] * inv;
+        codes[i * cstride] = oracle_e4m3_encode(y);
+    }
+    if (e8) *e8 = (uint8_t)(e + 127);
+    return ldexpf(1.0f, e);
+}
+
+/* A side: X is rows x cols (contracted axis = columns), blocks 1 x blk.
+ * codes: rows x cols; scales: rows x (cols/blk) */
+void oracle_quant_rows(const float *X, int64_t rows, int64_t cols, int64_t ld,
+                       int blk, int mode, float amax_floor,
+                       uint8_t *codes, float *scales, uint8_t *e8)
+{
+    qparams_t qp = { blk, mode, amax_floor };
+    int64_t nb = cols / blk;
+    for (int64_t i = 0; i < rows; ++i)
+        for (int64_t b = 0; b < nb; ++b)
+            scales[i * nb + b] = quant_block(X + i * ld + b * blk, 1, blk, &qp,
+                                             codes + i * cols + b * blk, 1,
+                                             e8 ? e8 + i * nb + b : NULL);
+}
+
+/* B side: X is rows x cols (contracted axis = rows), blocks blk x 1.
+ * codes: rows x cols; scales: (rows/blk) x cols */
+void oracle_quant_cols(const float *X, int64_t rows, int64_t cols, int64_t ld,
+                       int blk, int mode, float amax_floor,
+                       uint8_t *codes, float *scales, uint8_t *e8)
+{
+    qparams_t qp = { blk, mode, amax_floor };
+    int64_t nb = rows / blk;
+    for (int64_t b = 0; b < nb; ++b)
+        for (int64_t j = 0; j < cols; ++j)
+            scales[b * cols + j] = quant_block(X + b * blk * ld + j, ld, blk, &qp,
+                                               codes + b * blk * cols + j, cols,
+                                               e8 ? e8 + b * cols + j : NULL);
+}
+
+/* -------------------------------------------------- linear combinations */
+
+/* out = sum_j c[j] * X_j over the four quadrants of X (rows x cols, leading
+ * dimension ld), in fp32: zero coefficients skipped, first term a rounded
+ * multiply, the rest fused multiply-adds, quadrant order 11,12,21,22. */
+static void comb(const float c[4], const float *X, int64_t rows, int64_t cols, int64_t ld,
+                 float *out /* rows/2 x cols/2, dense */)
+{
+    int64_t hr = rows / 2, hc = cols / 2;
+    const float *Q[4] = { X, X + hc, X + hr * ld, X + hr * ld + hc };
+    for (int64_t i = 0; i < hr; ++i) {
+        for (int64_t k = 0; k < hc; ++k) {
+            float acc = 0.0f;
+            int set = 0;
+            for (int j = 0; j < 4; ++j) {
+                if (c[j] == 0.0f) continue;
+                float x = Q[j][i * ld + k];
+                if (!set) { acc = c[j] * x; set = 1; }
+                else acc = fmaf(c[j], x, acc);
+            }
+            out[i * hc + k] = acc;
+        }
+    }
+}
+
+/* ------------------------------------------------------------ fp64 GEMM */
+
+/* C (m x n, fp64) = A (m x k) * B (k x n), plain i-k-j loops.  This is the
+ * library-free definition of the product; rows are independent, so the outer
+ * loop may be spread over cores without changing any result. */
+static void gemm_f64(const double *A, const double *B, double *C,
+                     int64_t m, int64_t n, int64_t k)
+{
+#pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < m; ++i) {
+        double *c = C + i * n;
+        for (int64_t j = 0; j < n; ++j) c[j] = 0.0;
+        for (int64_t p = 0; p < k; ++p) {
+            double a = A[i * k + p];
+            const double *b = B + p * n;
+            for (int64_t j = 0; j < n; ++j) c[j] += a * b[j];
+        }
+    }
+}
+
+/* fp64 product of fp32 inputs: the "higher-precision reference" of App. E.2. */
+void oracle_ref_gemm(const float *A, const float *B, double *C,
+                     int64_t M, int64_t N, int64_t K)
+{
+    double *Ad = (double *)malloc(sizeof(double) * M * K);
+    double *Bd = (double *)malloc(sizeof(double) * K * N);
+    for (int64_t i = 0; i < M * K; ++i) Ad[i] = (double)A[i];
+    for (int64_t i = 0; i < K * N; ++i) Bd[i] = (double)B[i];
+    gemm_f64(Ad, Bd, C, M, N, K);
+    free(Ad); free(Bd);
+}
+
+/* Selected rows of the fp64 reference product (for sampled checks at sizes
+ * where the whole product is too slow): Crows[s, :] = A[rows[s], :] * B. */
+void oracle_ref_gemm_rows(const float *A, const float *B, const int64_t *rows, int64_t nrows,
+                          double *Crows, int64_t M, int64_t N, int64_t K)
+{
+    (void)M;
+#pragma omp parallel for schedule(static)
+    for (int64_t s = 0; s < nrows; ++s) {
+        double *c = Crows + s * N;
+        const float *a = A + rows[s] * K;
+        for (int64_t j = 0; j < N; ++j) c[j] = 0.0;
+        for (int64_t p = 0; p < K; ++p) {
+            double av = (double)a[p];
+            const float *b = B + p * N;
+            for (int64_t j = 0; j < N; ++j) c[j] += av * (double)b[j];
+        }
+    }
+}
+
+/* ---------------------------------------------------- fused fast matmul */
+
+typedef struct {
+    int rank;
+    float U[ORACLE_MAX_RANK][4], V[ORACLE_MAX_RANK][4], W[ORACLE_MAX_RANK][4];
+    qparams_t qp;
+} realization_t;
+
+/* Leaf: quantize both operands block-wise, dequantize exactly into fp64, multiply. */
+static void leaf_product(const float *A, int64_t lda, const float *B, int64_t ldb,
+                         int64_t m, int64_t n, int64_t k, const qparams_t *qp, double *C)
+{
+    double *Ad = (double *)malloc(sizeof(double) * m * k);
+    double *Bd = (double *)malloc(sizeof(double) * k * n);
+    if (qp->mode == SCALE_IDENTITY) {
+        for (int64_t i = 0; i < m; ++i)
+            for (int64_t p = 0; p < k; ++p) Ad[i * k + p] = (double)A[i * lda + p];
+        for (int64_t p = 0; p < k; ++p)
+            for (int64_t j = 0; j < n; ++j) Bd[p * n + j] = (double)B[p * ldb + j];
+    } else {
+        int64_t nb = k / qp->blk;
+        uint8_t *ca = (uint8_t *)malloc((size_t)(m * k));
+        float *sa = (float *)malloc(sizeof(float) * m * nb);
+        uint8_t *cb = (uint8_t *)malloc((size_t)(k * n));
+        float *sb = (float *)malloc(sizeof(float) * nb * n);
+        oracle_quant_rows(A, m, k, lda, qp->blk, qp->mode, qp->amax_floor, ca, sa, NULL);
+        oracle_quant_cols(B, k, n, ldb, qp->blk, qp->mode, qp->amax_floor, cb, sb, NULL);
+        for (int64_t i = 0; i < m; ++i)
+            for (int64_t p = 0; p < k; ++p)
+                Ad[i * k + p] = oracle_e4m3_decode(ca[i * k + p]) * (double)sa[i * nb + p / qp->blk];
+        for (int64_t p = 0; p < k; ++p)
+            for (int64_t j = 0; j < n; ++j)
+                Bd[p * n + j] = oracle_e4m3_decode(cb[p * n + j]) * (double)sb[(p / qp->blk) * n + j];
+        free(ca); free(sa); free(cb); free(sb);
+    }
+    gemm_f64(Ad, Bd, C, m, n, k);
+    free(Ad); free(Bd);
+}
+
+static void fused_rec(const realization_t *D, int levels,
+                      const float *A, int64_t lda, const float *B, int64_t ldb,
+                      int64_t m, int64_t n, int64_t k, double *C /* m x n dense */)
+{
+    if (levels == 0) { leaf_product(A, lda, B, ldb, m, n, k, &D->qp, C); return; }
+    int64_t hm = m / 2, hn = n / 2, hk = k / 2;
+    float *S = (float *)malloc(sizeof(float) * hm * hk);
+    float *T = (float *)malloc(sizeof(float) * hk * hn);
+    double *Mr = (double *)malloc(sizeof(double) * hm * hn);
+    int touched[4] = { 0, 0, 0, 0 };
+    for (int r = 0; r < D->rank; ++r) {
+        comb(D->U[r], A, m, k, lda, S);
+        comb(D->V[r], B, k, n, ldb, T);
+        fused_rec(D, levels - 1, S, hk, T, hn, hm, hn, hk, Mr);
+        for (int q = 0; q < 4; ++q) {
+            double w = (double)D->W[r][q];
+            if (w == 0.0) continue;
+            double *Cq = C + (q >> 1) * hm * n + (q & 1) * hn;
+            for (int64_t i = 0; i < hm; ++i)
+                for (int64_t j = 0; j < hn; ++j) {
+                    double v = w * Mr[i * hn + j];
+                    if (touched[q]) Cq[i * n + j] += v; else Cq[i * n + j] = v;
+                }
+            touched[q] = 1;
+        }
+    }
+    for (int q = 0; q < 4; ++q)
+        if (!touched[q]) {
+            double *Cq = C + (q >> 1) * hm * n + (q & 1) * hn;
+            for (int64_t i = 0; i < hm; ++i)
+                for (int64_t j = 0; j < hn; ++j) Cq[i * n + j] = 0.0;
+        }
+    free(S); free(T); free(Mr);
+}
+
+static void fill_realization(realization_t *D, int rank, const float *U, const float *V,
+                             const float *W, int blk, int mode, float amax_floor)
+{
+    memset(D, 0, sizeof(*D));
+    D->rank = rank;
+    for (int r = 0; r < rank; ++r)
+        for (int j = 0; j < 4; ++j) {
+            D->U[r][j] = U ? U[r * 4 + j] : 0.0f;
+            D->V[r][j] = V ? V[r * 4 + j] : 0.0f;
+            D->W[r][j] = W ? W[r * 4 + j] : 0.0f;
+        }
+    D->qp.blk = blk; D->qp.mode = mode; D->qp.amax_floor = amax_floor;
+}
+
+/* C (fp64, M x N) = fused block-scaled fast product of A (M x K) and B (K x N).
+ * levels == 0 is the cubic fp8 product (U, V, W unused).  Returns 0 on success. */
+int oracle_fused_fmm(const float *A, const float *B, double *C,
+                     int64_t M, int64_t N, int64_t K,
+                     int rank, const float *U, const float *V, const float *W,
+                     int levels, int blk, int mode, float amax_floor)
+{
+    if (rank > ORACLE_MAX_RANK || levels < 0) return 1;
+    int64_t div = (int64_t)1 << levels;
+    if (M % div || N % div || K % div) return 2;
+    if (mode != SCALE_IDENTITY && (K / div) % blk) return 3;
+    realization_t D;
+    fill_realization(&D, rank, U, V, W, blk, mode, amax_floor);
+    fused_rec(&D, levels, A, K, B, N, M, N, K, C);
+    return 0;
+}
+
+/* ------------------------------- quantized leaf operands, for bit parity */
+
+static void encode_rec(const realization_t *D, int levels, int side,
+                       const float *X, int64_t ld, int64_t rows, int64_t cols,
+                       int64_t *term, uint8_t *codes, float *scales, uint8_t *e8)
+{
+    if (levels == 0) {
+        int64_t nb = (side == 0 ? cols : rows) / D->qp.blk;
+        int64_t nsc = side == 0 ? rows * nb : nb * cols;
+        uint8_t *c = codes + *term * rows * cols;
+        float *s = scales + *term * nsc;
+        uint8_t *e = e8 ? e8 + *term * nsc : NULL;
+        if (side == 0) oracle_quant_rows(X, rows, cols, ld, D->qp.blk, D->qp.mode, D->qp.amax_floor, c, s, e);
+        else           oracle_quant_cols(X, rows, cols, ld, D->qp.blk, D->qp.mode, D->qp.amax_floor, c, s, e);
+        *term += 1;
+        return;
+    }
+    float *S = (float *)malloc(sizeof(float) * (rows / 2) * (cols / 2));
+    for (int r = 0; r < D->rank; ++r) {
+        comb(side == 0 ? D->U[r] : D->V[r], X, rows, cols, ld, S);
+        encode_rec(D, levels - 1, side, S, cols / 2, rows / 2, cols / 2, term, codes, scales, e8);
+    }
+    free(S);
+}
+
+/* Quantized leaf operands of one side, terms in depth-first order
+ * t = (r_1 * R + r_2) * R + ... (r_1 = outermost level).
+ * side 0: X = A (M x K): codes [T][M/2^l][K/2^l], scales [T][M/2^l][K/2^l/blk]
+ * side 1: X = B (K x N): codes [T][K/2^l][N/2^l], scales [T][K/2^l/blk][N/2^l]
+ * e8 (may be NULL): biased UE8M0 exponent bytes, same shape as scales. */
+int oracle_encode(const float *X, int64_t rows, int64_t cols, int side,
+                  int rank, const float *U, const float *V,
+                  int levels, int blk, int mode, float amax_floor,
+                  uint8_t *codes, float *scales, uint8_t *e8)
+{
+    if (rank > ORACLE_MAX_RANK || levels < 0 || mode == SCALE_IDENTITY) return 1;
+    int64_t div = (int64_t)1 << levels;
+    if (rows % div || cols % div) return 2;
+    if (((side == 0 ? cols : rows) / div) % blk) return 3;
+    realization_t D;
+    fill_realization(&D, rank, U, V, NULL, blk, mode, amax_floor);
+    int64_t term = 0;
+    encode_rec(&D, levels, side, X, cols, rows, cols, &term, codes, scales, e8);
+    return 0;
+}
+
+/* ----------------------------------------------------------- error stats */
+
+/* out[0] = sum (C - Cref)^2, out[1] = sum Cref^2, out[2] = max |C - Cref| */
+void oracle_error_stats(const double *C, const double *Cref, int64_t count, double *out)
+{
+    double sd = 0.0, sr = 0.0, mx = 0.0;
+    for (int64_t i = 0; i < count; ++i) {
+        double d = C[i] - Cref[i];
+        sd += d * d;
+        sr += Cref[i] * Cref[i];
+        if (fabs(d) > mx) mx = fabs(d);
+    }
+    out[0] = sd; out[1] = sr; out[2] = mx;
+}
+
+int oracle_num_threads(void)
+{
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
