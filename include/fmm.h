@@ -1,0 +1,160 @@
+/*
+ * fmm.h - C ABI of the B200 (sm_100a) library for block-scaled e4m3 fast matrix
+ * multiplication  C = A * B  through a rank-R 2x2 realization (U, V, W).
+ *
+ * The operation (paper Sec. 2.1-2.2, App. D.1, App. E.2):
+ *   split A (M x K) and B (K x N) into 2x2 blocks, row-vectorised in the order
+ *   11, 12, 21, 22; for every term r form the encoded combinations
+ *       S_r = sum_j U[r][j] A_j ,   T_r = sum_j V[r][j] B_j          (fp32)
+ *   quantize S_r and T_r to e4m3 per block of `block_k` consecutive elements along
+ *   the contracted axis (one scale per block, both sides), multiply the quantized
+ *   operands with fp32 accumulation, and decode
+ *       C_q = sum_r W[r][q] * (S_r^ * T_r^) .
+ *   The raw operands are never quantized.  With `levels` > 1 the encoders and the
+ *   decoder are applied recursively (Kronecker power) and only the R^levels leaf
+ *   combinations are quantized (Sec. 3).  levels == 0 is the cubic fp8 product:
+ *   A and B themselves are quantized and multiplied once.
+ *
+ * General rules
+ *   - Every function returns fmm_status_t; nothing throws, aborts or traps the device.
+ *   - "dev" pointers are device pointers of the current CUDA device, "host" pointers are
+ *     host memory.  The caller owns every buffer it passes.  fmm_matmul, fmm_encode_only,
+ *     fmm_ref_gemm_fp64 and fmm_error_stats allocate nothing and only enqueue work on
+ *     `cuda_stream` (a cudaStream_t passed as void*; NULL = default stream); they do not
+ *     synchronise.  Inputs must be finite.
+ *   - All matrices are dense row-major with no padding.
+ *   - There is no CPU fallback: on a machine without a B200-class device the device
+ *     functions return FMM_ERR_CUDA or FMM_ERR_ARCH.
+ */
+#ifndef FMM_B200_H
+#define FMM_B200_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    FMM_OK = 0,
+    FMM_ERR_INVALID_ARG = 1,    /* null pointer, bad enum, bad rank / levels / block size */
+    FMM_ERR_SHAPE = 2,          /* M, N, K not divisible as required (see fmm_matmul) */
+    FMM_ERR_NOT_EXACT = 3,      /* (U, V, W) violates the Brent equations beyond 1e-5 */
+    FMM_ERR_WORKSPACE = 4,      /* workspace missing, misaligned or too small */
+    FMM_ERR_ALLOC = 5,          /* host or device allocation failed (plan creation only) */
+    FMM_ERR_CUDA = 6,           /* a CUDA runtime / driver call failed (no device, bad stream, ...) */
+    FMM_ERR_ARCH = 7,           /* current device is not compute capability 10.x */
+    FMM_ERR_DEVICE_TIMEOUT = 8  /* a bounded device-side wait gave up (see fmm_device_status) */
+} fmm_status_t;
+
+typedef enum {
+    /* Paper's quantizer (App. E.2): scale = amax / 448 kept in fp32. */
+    FMM_SCALE_FP32_AMAX_DIV_448 = 0,
+    /* Hardware-native deviation from the paper: the scale is rounded UP to a power of two
+     * (UE8M0, e = ceil(log2(amax/448))) so that the tensor cores apply it themselves.
+     * Requires block_k == 32.  Every number produced in this mode must be labelled as such. */
+    FMM_SCALE_UE8M0_CEIL = 1
+} fmm_scale_mode_t;
+
+typedef struct {
+    int block_k;                 /* 32 or 128: block length along the contracted axis */
+    fmm_scale_mode_t scale_mode;
+    float amax_floor;            /* minimum-scale clamp on the block amax; the paper uses 1e-12 */
+    float fp8_max;               /* largest e4m3 magnitude; must be 448 */
+} fmm_quant_params_t;
+
+typedef struct fmm_plan fmm_plan_t;   /* opaque */
+
+/* Create a plan on the current CUDA device (Sec. 2.1: a realization is three R x 4 arrays).
+ *   rank    number of terms R, 1..8 (7 for Strassen-type realizations, 8 for the cubic one);
+ *           ignored when levels == 0.
+ *   U, V, W host, rank x 4 row-major fp32, column order 11, 12, 21, 22.  W[r][q] is the weight of
+ *           product r in output block C_q in that same order (NOT the paper's cyclic third
+ *           factor w_r = rv(W_r^T); swap entries 12 and 21 to convert).  May be NULL when levels == 0.
+ *   levels  0 (cubic fp8) .. 3.
+ *   qp      quantizer parameters (copied).
+ * Checks the Brent equations in fp64 (max residual <= 1e-5 else FMM_ERR_NOT_EXACT).  Allocates a few
+ * KB of device memory for term tables and a status word; freed by fmm_plan_destroy. */
+fmm_status_t fmm_plan_create(fmm_plan_t** plan, int rank, const float* U, const float* V,
+                             const float* W, int levels, const fmm_quant_params_t* qp);
+fmm_status_t fmm_plan_destroy(fmm_plan_t* plan);
+
+/* Bytes of device workspace fmm_matmul / fmm_encode_only need for this problem size (host call).
+ * The workspace holds the quantized leaf operands, their scales and, for levels >= 2, the fp32
+ * intermediate combinations of the outer levels. */
+fmm_status_t fmm_workspace_bytes(const fmm_plan_t* plan, int64_t M, int64_t N, int64_t K,
+                                 size_t* bytes);
+
+/* C = A * B through the plan's realization (whole hot path: pre-addition + quantization of both
+ * sides, the R^levels block-scaled fp8 products on the tensor cores, post-addition into C).
+ *   A dev, M x K fp32;  B dev, K x N fp32;  C dev, M x N fp32, overwritten.
+ *   Shape rule: with d = 2^levels, M/d and N/d must be multiples of 128 and K/d a multiple of 128
+ *   (hence of block_k); otherwise FMM_ERR_SHAPE.
+ *   workspace dev, 1024-byte aligned, at least fmm_workspace_bytes() bytes, caller-owned; its
+ *   contents after the call are the quantized operands (see fmm_quantized_view).
+ * Asynchronous on cuda_stream.  Calls sharing a plan or a workspace must be stream-ordered. */
+fmm_status_t fmm_matmul(const fmm_plan_t* plan, const float* A, const float* B, float* C,
+                        int64_t M, int64_t N, int64_t K, void* workspace, size_t workspace_bytes,
+                        void* cuda_stream);
+
+/* Steps 1-2 only (pre-addition + quantization of both sides) into the workspace. */
+fmm_status_t fmm_encode_only(const fmm_plan_t* plan, const float* A, const float* B,
+                             int64_t M, int64_t N, int64_t K, void* workspace,
+                             size_t workspace_bytes, void* cuda_stream);
+
+/* The tensor-core products + post-addition only, on operands a previous fmm_encode_only /
+ * fmm_matmul left in the workspace. */
+fmm_status_t fmm_multiply_only(const fmm_plan_t* plan, float* C, int64_t M, int64_t N, int64_t K,
+                               void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* Where the quantized leaf operand of term `term` (depth-first order t = (r1*R + r2)*R + ...,
+ * r1 = outermost level; 0 for levels == 0) lives in the workspace (host call, byte offsets).
+ *   side 'A': codes are q_rows x q_cols = (M/d) x (K/d) e4m3 bytes, row-major (K contiguous).
+ *   side 'B': codes are stored TRANSPOSED, q_rows x q_cols = (N/d) x (K/d) (K contiguous).
+ *   FP32 scale mode: fp32 scales; side 'A': scale_rows x scale_cols = (M/d) x (K/d/block_k) row-major;
+ *             side 'B': (K/d/block_k) x (N/d) row-major.
+ *   UE8M0 mode: one biased-exponent byte per block in 512-byte tiles of 128 rows x 4 blocks:
+ *             tile index (row/128) * (nblocks/4) + (block/4), byte (row%32)*16 + ((row%128)/32)*4 + block%4
+ *             where row is the M/d (side 'A') or N/d (side 'B') index; scale_rows x scale_cols then
+ *             report that logical (rows x blocks) shape. */
+fmm_status_t fmm_quantized_view(const fmm_plan_t* plan, int64_t M, int64_t N, int64_t K, int term,
+                                char side, size_t* q_offset, int64_t* q_rows, int64_t* q_cols,
+                                size_t* scale_offset, int64_t* scale_rows, int64_t* scale_cols);
+
+/* Higher-precision reference of App. E.2: Cref (dev, M x N fp64) = A * B with fp64 accumulation of
+ * the fp32 inputs (dev).  M, N multiples of 64; K a multiple of 16.  Off the timed path. */
+fmm_status_t fmm_ref_gemm_fp64(const float* A, const float* B, double* Cref,
+                               int64_t M, int64_t N, int64_t K, void* cuda_stream);
+
+/* Error statistics of App. E.2 / Eq. (D.9): out3 (dev, 3 doubles) =
+ * [ sum (C - Cref)^2, sum Cref^2, max |C - Cref| ] over the M x N entries; the relative Frobenius
+ * error is sqrt(out3[0] / out3[1]).  Overwrites out3; deterministic (no floating-point atomics).
+ * scratch: dev, at least fmm_error_stats_scratch_bytes() bytes, caller-owned. */
+fmm_status_t fmm_error_stats(const float* C, const double* Cref, int64_t M, int64_t N,
+                             double* out3, void* scratch, size_t scratch_bytes, void* cuda_stream);
+size_t fmm_error_stats_scratch_bytes(void);
+
+/* Reads the plan's device status word (synchronises the device).  *code == 0: no bounded wait has
+ * given up since plan creation; otherwise a kernel-specific location code, and the results of the
+ * call that set it are invalid.  Returns FMM_ERR_DEVICE_TIMEOUT when *code != 0. */
+fmm_status_t fmm_device_status(const fmm_plan_t* plan, int* code);
+
+/* Host utility (Sec. 2.1): Phi = sum_r |U_r|^2 |V_r|^2 |W_r|^2 and Gamma = sum_r |U_r| |V_r| |W_r|
+ * with entrywise 2-norms, in fp64. */
+fmm_status_t fmm_phi_gamma(int rank, const float* U, const float* V, const float* W,
+                           double* phi, double* gamma);
+
+/* Host utility: largest absolute residual of the 64 Brent equations of <2,2,2>, in fp64. */
+fmm_status_t fmm_brent_residual(int rank, const float* U, const float* V, const float* W,
+                                double* max_residual);
+
+/* Number of kernels the last fmm_matmul / fmm_encode_only / fmm_multiply_only on this plan launched. */
+fmm_status_t fmm_last_launch_count(const fmm_plan_t* plan, int* launches);
+
+const char* fmm_status_string(fmm_status_t status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FMM_B200_H */

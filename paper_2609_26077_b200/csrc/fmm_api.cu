@@ -1,0 +1,383 @@
+// Host side of the C ABI: plan validation, workspace layout, the recursion driver that turns
+// (levels, realization) into kernel launches.  No device allocation happens after plan creation.
+#include <math.h>
+#include <stdlib.h>
+#include <string.h>
+#include <new>
+#include <vector>
+#include "fmm_internal.h"
+
+namespace {
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+bool finite_all(const float* p, int n)
+{
+    for (int i = 0; i < n; ++i)
+        if (!isfinite(p[i])) return false;
+    return true;
+}
+
+// Largest residual of the Brent equations of <2,2,2> (Sec. 2.1: the decomposition must equal the
+// matrix-multiplication tensor): sum_r U[r][ij] V[r][kl] W[r][mn] = [j==k][i==m][l==n].
+double brent_residual(int rank, const float* U, const float* V, const float* W)
+{
+    double worst = 0.0;
+    for (int a = 0; a < 4; ++a)
+        for (int b = 0; b < 4; ++b)
+            for (int c = 0; c < 4; ++c) {
+                double s = 0.0;
+                for (int r = 0; r < rank; ++r)
+                    s += (double)U[r * 4 + a] * (double)V[r * 4 + b] * (double)W[r * 4 + c];
+                const int i = a >> 1, j = a & 1, k = b >> 1, l = b & 1, m = c >> 1, n = c & 1;
+                const double target = (j == k && i == m && l == n) ? 1.0 : 0.0;
+                worst = fmax(worst, fabs(s - target));
+            }
+    return worst;
+}
+
+fmm_status_t check_shape(const fmm_plan* plan, int64_t M, int64_t N, int64_t K)
+{
+    if (M <= 0 || N <= 0 || K <= 0) return FMM_ERR_SHAPE;
+    const int64_t d = (int64_t)1 << plan->levels;
+    if (M % d || N % d || K % d) return FMM_ERR_SHAPE;
+    if ((M / d) % 128 || (N / d) % 128 || (K / d) % 128) return FMM_ERR_SHAPE;
+    if (M > (1 << 30) || N > (1 << 30) || K > (1 << 30)) return FMM_ERR_SHAPE;
+    return FMM_OK;
+}
+
+void make_layout(const fmm_plan* plan, int64_t M, int64_t N, int64_t K, FmmLayout* L)
+{
+    const int64_t d = (int64_t)1 << plan->levels;
+    L->m = M / d; L->n = N / d; L->k = K / d;
+    L->terms = plan->terms;
+    const int64_t nkb = L->k / plan->qp.block_k;
+    size_t off = 0;
+    L->qa = off; off = align_up(off + (size_t)(L->terms * L->m * L->k), 1024);
+    L->qb = off; off = align_up(off + (size_t)(L->terms * L->n * L->k), 1024);
+    const size_t sbytes = plan->qp.scale_mode == FMM_SCALE_FP32_AMAX_DIV_448 ? 4 : 1;
+    L->sa_term = (size_t)(L->m * nkb) * sbytes;
+    L->sb_term = (size_t)(L->n * nkb) * sbytes;
+    L->sa = off; off = align_up(off + L->sa_term * L->terms, 1024);
+    L->sb = off; off = align_up(off + L->sb_term * L->terms, 1024);
+    for (int lv = 0; lv < FMM_MAX_LEVELS; ++lv) { L->inter_a[lv] = 0; L->inter_b[lv] = 0; }
+    // fp32 combinations of the outer levels 1 .. levels-1
+    for (int lv = 1; lv < plan->levels; ++lv) {
+        const int64_t cnt = fmm_ipow(plan->rank, lv);
+        const int64_t dd = (int64_t)1 << lv;
+        L->inter_a[lv] = off; off = align_up(off + (size_t)(cnt * (M / dd) * (K / dd)) * 4, 1024);
+        L->inter_b[lv] = off; off = align_up(off + (size_t)(cnt * (K / dd) * (N / dd)) * 4, 1024);
+    }
+    L->total = off;
+}
+
+fmm_status_t check_ws(const fmm_plan* plan, int64_t M, int64_t N, int64_t K, void* ws, size_t ws_bytes,
+                      FmmLayout* L)
+{
+    fmm_status_t s = check_shape(plan, M, N, K);
+    if (s != FMM_OK) return s;
+    make_layout(plan, M, N, K, L);
+    if (!ws || ((uintptr_t)ws & 1023) || ws_bytes < L->total) return FMM_ERR_WORKSPACE;
+    return FMM_OK;
+}
+
+void fill_coef(float dst[FMM_MAX_RANK][4], const float src[FMM_MAX_RANK][4], int R)
+{
+    memset(dst, 0, sizeof(float) * FMM_MAX_RANK * 4);
+    for (int r = 0; r < R; ++r)
+        for (int j = 0; j < 4; ++j) dst[r][j] = src[r][j];
+}
+
+// One side of steps 1-2: outer levels as fp32 combinations, last level fused with the quantizer.
+fmm_status_t encode_side(fmm_plan* plan, const FmmLayout& L, char* ws, const float* X,
+                         int64_t rows, int64_t cols, bool b_side, cudaStream_t st)
+{
+    const int R = plan->rank, lv = plan->levels;
+    const int blk = plan->qp.block_k, mode = (int)plan->qp.scale_mode;
+    const float (*coef)[4] = b_side ? plan->V : plan->U;
+    EncodeParams e;
+    memset(&e, 0, sizeof(e));
+    e.q_out = reinterpret_cast<uint8_t*>(ws + (b_side ? L.qb : L.qa));
+    e.s_out = ws + (b_side ? L.sb : L.sa);
+    e.s_term_stride = (int64_t)(b_side ? L.sb_term : L.sa_term);
+    e.amax_floor = plan->qp.amax_floor;
+    fmm_status_t s;
+    if (lv == 0) {
+        e.in = X; e.in_batch_stride = 0; e.ld = cols; e.batch = 1;
+        e.rows = (int)rows; e.cols = (int)cols; e.nq = 1; e.R = 1;
+        e.coef[0][0] = 1.0f;
+    } else {
+        const float* cur = X;
+        int64_t cur_rows = rows, cur_cols = cols, cur_ld = cols, cur_stride = 0;
+        int batch = 1;
+        for (int level = 1; level < lv; ++level) {
+            CombParams c;
+            memset(&c, 0, sizeof(c));
+            c.in = cur; c.in_batch_stride = cur_stride; c.ld = cur_ld; c.batch = batch;
+            c.rows = (int)(cur_rows / 2); c.cols = (int)(cur_cols / 2); c.R = R;
+            fill_coef(c.coef, coef, R);
+            c.out = reinterpret_cast<float*>(ws + (b_side ? L.inter_b[level] : L.inter_a[level]));
+            s = fmm_launch_comb(c, st);
+            if (s != FMM_OK) return s;
+            plan->last_launches++;
+            cur = c.out; cur_rows /= 2; cur_cols /= 2; cur_ld = cur_cols; cur_stride = cur_rows * cur_cols;
+            batch *= R;
+        }
+        e.in = cur; e.in_batch_stride = cur_stride; e.ld = cur_ld; e.batch = batch;
+        e.rows = (int)(cur_rows / 2); e.cols = (int)(cur_cols / 2); e.nq = 4; e.R = R;
+        fill_coef(e.coef, coef, R);
+    }
+    s = b_side ? fmm_launch_encode_b(e, blk, mode, st) : fmm_launch_encode_a(e, blk, mode, st);
+    if (s == FMM_OK) plan->last_launches++;
+    return s;
+}
+
+fmm_status_t multiply(fmm_plan* plan, const FmmLayout& L, char* ws, float* C, int64_t M, int64_t N,
+                      cudaStream_t st)
+{
+    GemmParams g;
+    memset(&g, 0, sizeof(g));
+    g.qa = reinterpret_cast<const uint8_t*>(ws + L.qa);
+    g.qb = reinterpret_cast<const uint8_t*>(ws + L.qb);
+    g.sa = ws + L.sa; g.sb = ws + L.sb;
+    g.sa_term = (int64_t)L.sa_term; g.sb_term = (int64_t)L.sb_term;
+    g.C = C; g.ldc = N; g.Mfull = M; g.Nfull = N;
+    g.m = (int)L.m; g.n = (int)L.n; g.k = (int)L.k; g.terms = (int)L.terms;
+    g.out_start = plan->d_out_start; g.out = plan->d_out; g.status = plan->d_status;
+    int launches = 0;
+    fmm_status_t s = fmm_launch_gemm(g, plan->qp.block_k, (int)plan->qp.scale_mode, st, &launches);
+    plan->last_launches += launches;
+    return s;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* fmm_status_string(fmm_status_t s)
+{
+    switch (s) {
+        case FMM_OK: return "ok";
+        case FMM_ERR_INVALID_ARG: return "invalid argument";
+        case FMM_ERR_SHAPE: return "shape not supported (M, N, K must be 2^levels * multiples of 128)";
+        case FMM_ERR_NOT_EXACT: return "realization violates the Brent equations";
+        case FMM_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+        case FMM_ERR_ALLOC: return "allocation failed";
+        case FMM_ERR_CUDA: return "CUDA call failed";
+        case FMM_ERR_ARCH: return "device is not compute capability 10.x (B200)";
+        case FMM_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait timed out";
+    }
+    return "unknown status";
+}
+
+fmm_status_t fmm_phi_gamma(int rank, const float* U, const float* V, const float* W, double* phi, double* gamma)
+{
+    if (rank < 1 || rank > FMM_MAX_RANK || !U || !V || !W || !phi || !gamma) return FMM_ERR_INVALID_ARG;
+    double p = 0.0, g = 0.0;
+    for (int r = 0; r < rank; ++r) {
+        double nu = 0, nv = 0, nw = 0;
+        for (int j = 0; j < 4; ++j) {
+            nu += (double)U[r * 4 + j] * U[r * 4 + j];
+            nv += (double)V[r * 4 + j] * V[r * 4 + j];
+            nw += (double)W[r * 4 + j] * W[r * 4 + j];
+        }
+        p += nu * nv * nw;
+        g += sqrt(nu * nv * nw);
+    }
+    *phi = p; *gamma = g;
+    return FMM_OK;
+}
+
+fmm_status_t fmm_brent_residual(int rank, const float* U, const float* V, const float* W, double* out)
+{
+    if (rank < 1 || rank > FMM_MAX_RANK || !U || !V || !W || !out) return FMM_ERR_INVALID_ARG;
+    *out = brent_residual(rank, U, V, W);
+    return FMM_OK;
+}
+
+fmm_status_t fmm_plan_create(fmm_plan_t** out, int rank, const float* U, const float* V, const float* W,
+                             int levels, const fmm_quant_params_t* qp)
+{
+    if (!out) return FMM_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (!qp || levels < 0 || levels > FMM_MAX_LEVELS) return FMM_ERR_INVALID_ARG;
+    if (qp->block_k != 32 && qp->block_k != 128) return FMM_ERR_INVALID_ARG;
+    if (qp->scale_mode != FMM_SCALE_FP32_AMAX_DIV_448 && qp->scale_mode != FMM_SCALE_UE8M0_CEIL) return FMM_ERR_INVALID_ARG;
+    if (qp->scale_mode == FMM_SCALE_UE8M0_CEIL && qp->block_k != 32) return FMM_ERR_INVALID_ARG;
+    if (qp->fp8_max != 448.0f || !(qp->amax_floor > 0.0f) || !isfinite(qp->amax_floor)) return FMM_ERR_INVALID_ARG;
+    if (levels > 0) {
+        if (rank < 1 || rank > FMM_MAX_RANK || !U || !V || !W) return FMM_ERR_INVALID_ARG;
+        if (!finite_all(U, rank * 4) || !finite_all(V, rank * 4) || !finite_all(W, rank * 4)) return FMM_ERR_INVALID_ARG;
+        if (brent_residual(rank, U, V, W) > 1e-5) return FMM_ERR_NOT_EXACT;
+    } else {
+        rank = 1;
+    }
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return FMM_ERR_CUDA; }
+    int major = 0;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) { cudaGetLastError(); return FMM_ERR_CUDA; }
+    if (major != 10) return FMM_ERR_ARCH;
+
+    fmm_plan* p = new (std::nothrow) fmm_plan;
+    if (!p) return FMM_ERR_ALLOC;
+    memset(p, 0, sizeof(*p));
+    p->rank = rank; p->levels = levels; p->qp = *qp; p->device = dev;
+    if (levels > 0)
+        for (int r = 0; r < rank; ++r)
+            for (int j = 0; j < 4; ++j) { p->U[r][j] = U[r * 4 + j]; p->V[r][j] = V[r * 4 + j]; p->W[r][j] = W[r * 4 + j]; }
+    p->terms = (int)fmm_ipow(rank, levels);
+
+    // Decoder table: destinations of every leaf product (Sec. 2.1 decode; Kronecker power for levels > 1).
+    const int nb = 1 << levels;                       // leaf blocks per side of C
+    std::vector<int> start(p->terms + 1, 0);
+    std::vector<FmmOutEntry> entries;
+    std::vector<char> touched((size_t)nb * nb, 0);
+    for (int t = 0; t < p->terms; ++t) {
+        start[t] = (int)entries.size();
+        int digits[FMM_MAX_LEVELS] = {0, 0, 0};
+        int tt = t;
+        for (int l = levels - 1; l >= 0; --l) { digits[l] = tt % rank; tt /= rank; }
+        const int paths = 1 << (2 * levels);
+        for (int path = 0; path < paths; ++path) {
+            double w = 1.0;
+            int rb = 0, cb = 0;
+            for (int l = 0; l < levels; ++l) {
+                const int q = (path >> (2 * (levels - 1 - l))) & 3;
+                w *= (double)p->W[digits[l]][q];
+                rb = rb * 2 + (q >> 1);
+                cb = cb * 2 + (q & 1);
+            }
+            if (levels == 0) { w = 1.0; }
+            if (w == 0.0) continue;
+            FmmOutEntry e;
+            e.row_off = rb; e.col_off = cb; e.w = (float)w;
+            e.first = touched[(size_t)rb * nb + cb] ? 0 : 1;
+            touched[(size_t)rb * nb + cb] = 1;
+            entries.push_back(e);
+        }
+    }
+    start[p->terms] = (int)entries.size();
+    p->n_out_total = (int)entries.size();
+
+    cudaError_t ce = cudaMalloc(&p->d_status, 4 * sizeof(int));
+    if (ce == cudaSuccess) ce = cudaMalloc(&p->d_out_start, sizeof(int) * start.size());
+    if (ce == cudaSuccess) ce = cudaMalloc(&p->d_out, sizeof(FmmOutEntry) * (entries.size() + 1));
+    if (ce == cudaSuccess) ce = cudaMemset(p->d_status, 0, 4 * sizeof(int));
+    if (ce == cudaSuccess) ce = cudaMemcpy(p->d_out_start, start.data(), sizeof(int) * start.size(), cudaMemcpyHostToDevice);
+    if (ce == cudaSuccess && !entries.empty())
+        ce = cudaMemcpy(p->d_out, entries.data(), sizeof(FmmOutEntry) * entries.size(), cudaMemcpyHostToDevice);
+    if (ce != cudaSuccess) {
+        cudaGetLastError();
+        fmm_plan_destroy(p);
+        return ce == cudaErrorMemoryAllocation ? FMM_ERR_ALLOC : FMM_ERR_CUDA;
+    }
+    *out = p;
+    return FMM_OK;
+}
+
+fmm_status_t fmm_plan_destroy(fmm_plan_t* p)
+{
+    if (!p) return FMM_ERR_INVALID_ARG;
+    if (p->d_status) cudaFree(p->d_status);
+    if (p->d_out_start) cudaFree(p->d_out_start);
+    if (p->d_out) cudaFree(p->d_out);
+    delete p;
+    return FMM_OK;
+}
+
+fmm_status_t fmm_workspace_bytes(const fmm_plan_t* plan, int64_t M, int64_t N, int64_t K, size_t* bytes)
+{
+    if (!plan || !bytes) return FMM_ERR_INVALID_ARG;
+    fmm_status_t s = check_shape(plan, M, N, K);
+    if (s != FMM_OK) return s;
+    FmmLayout L;
+    make_layout(plan, M, N, K, &L);
+    *bytes = L.total;
+    return FMM_OK;
+}
+
+fmm_status_t fmm_quantized_view(const fmm_plan_t* plan, int64_t M, int64_t N, int64_t K, int term, char side,
+                                size_t* q_offset, int64_t* q_rows, int64_t* q_cols,
+                                size_t* scale_offset, int64_t* scale_rows, int64_t* scale_cols)
+{
+    if (!plan || !q_offset || !q_rows || !q_cols || !scale_offset || !scale_rows || !scale_cols) return FMM_ERR_INVALID_ARG;
+    if (side != 'A' && side != 'B') return FMM_ERR_INVALID_ARG;
+    fmm_status_t s = check_shape(plan, M, N, K);
+    if (s != FMM_OK) return s;
+    if (term < 0 || term >= plan->terms) return FMM_ERR_INVALID_ARG;
+    FmmLayout L;
+    make_layout(plan, M, N, K, &L);
+    const int64_t nkb = L.k / plan->qp.block_k;
+    const bool fp32 = plan->qp.scale_mode == FMM_SCALE_FP32_AMAX_DIV_448;
+    if (side == 'A') {
+        *q_offset = L.qa + (size_t)term * L.m * L.k; *q_rows = L.m; *q_cols = L.k;
+        *scale_offset = L.sa + (size_t)term * L.sa_term; *scale_rows = L.m; *scale_cols = nkb;
+    } else {
+        *q_offset = L.qb + (size_t)term * L.n * L.k; *q_rows = L.n; *q_cols = L.k;
+        *scale_offset = L.sb + (size_t)term * L.sb_term;
+        if (fp32) { *scale_rows = nkb; *scale_cols = L.n; } else { *scale_rows = L.n; *scale_cols = nkb; }
+    }
+    return FMM_OK;
+}
+
+fmm_status_t fmm_encode_only(const fmm_plan_t* cplan, const float* A, const float* B, int64_t M, int64_t N, int64_t K,
+                             void* ws, size_t ws_bytes, void* stream)
+{
+    if (!cplan || !A || !B) return FMM_ERR_INVALID_ARG;
+    fmm_plan* plan = const_cast<fmm_plan*>(cplan);
+    FmmLayout L;
+    fmm_status_t s = check_ws(plan, M, N, K, ws, ws_bytes, &L);
+    if (s != FMM_OK) return s;
+    plan->last_launches = 0;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    s = encode_side(plan, L, static_cast<char*>(ws), A, M, K, false, st);
+    if (s != FMM_OK) return s;
+    return encode_side(plan, L, static_cast<char*>(ws), B, K, N, true, st);
+}
+
+fmm_status_t fmm_multiply_only(const fmm_plan_t* cplan, float* C, int64_t M, int64_t N, int64_t K,
+                               void* ws, size_t ws_bytes, void* stream)
+{
+    if (!cplan || !C) return FMM_ERR_INVALID_ARG;
+    fmm_plan* plan = const_cast<fmm_plan*>(cplan);
+    FmmLayout L;
+    fmm_status_t s = check_ws(plan, M, N, K, ws, ws_bytes, &L);
+    if (s != FMM_OK) return s;
+    plan->last_launches = 0;
+    return multiply(plan, L, static_cast<char*>(ws), C, M, N, reinterpret_cast<cudaStream_t>(stream));
+}
+
+fmm_status_t fmm_matmul(const fmm_plan_t* cplan, const float* A, const float* B, float* C,
+                        int64_t M, int64_t N, int64_t K, void* ws, size_t ws_bytes, void* stream)
+{
+    if (!cplan || !A || !B || !C) return FMM_ERR_INVALID_ARG;
+    fmm_plan* plan = const_cast<fmm_plan*>(cplan);
+    FmmLayout L;
+    fmm_status_t s = check_ws(plan, M, N, K, ws, ws_bytes, &L);
+    if (s != FMM_OK) return s;
+    plan->last_launches = 0;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    s = encode_side(plan, L, static_cast<char*>(ws), A, M, K, false, st);
+    if (s != FMM_OK) return s;
+    s = encode_side(plan, L, static_cast<char*>(ws), B, K, N, true, st);
+    if (s != FMM_OK) return s;
+    return multiply(plan, L, static_cast<char*>(ws), C, M, N, st);
+}
+
+fmm_status_t fmm_device_status(const fmm_plan_t* plan, int* code)
+{
+    if (!plan || !code) return FMM_ERR_INVALID_ARG;
+    int h[4] = {0, 0, 0, 0};
+    if (cudaMemcpy(h, plan->d_status, sizeof(h), cudaMemcpyDeviceToHost) != cudaSuccess) { cudaGetLastError(); return FMM_ERR_CUDA; }
+    *code = h[0];
+    return h[0] ? FMM_ERR_DEVICE_TIMEOUT : FMM_OK;
+}
+
+fmm_status_t fmm_last_launch_count(const fmm_plan_t* plan, int* launches)
+{
+    if (!plan || !launches) return FMM_ERR_INVALID_ARG;
+    *launches = plan->last_launches;
+    return FMM_OK;
+}
+
+}  // extern "C"

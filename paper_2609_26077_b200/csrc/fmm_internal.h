@@ -1,0 +1,83 @@
+// Internal declarations shared by the translation units of the library (not part of the C ABI).
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda.h>
+#include <stdint.h>
+#include "../../include/fmm.h"
+
+#define FMM_MAX_RANK 8
+#define FMM_MAX_LEVELS 3
+
+// One destination of a leaf product in C: block origin, weight, and whether this is the first
+// product written there (store) or a later one (accumulate).
+struct FmmOutEntry {
+    int row_off;   // element row of the destination block origin in C
+    int col_off;   // element column
+    float w;       // product of the W coefficients along the recursion path
+    int first;     // 1: overwrite, 0: add
+};
+
+struct FmmLayout {            // byte offsets into the workspace
+    int64_t m, n, k;          // leaf dimensions
+    int64_t terms;            // R^levels (1 for levels == 0)
+    size_t qa, qb;            // e4m3 codes, terms x m x k and terms x n x k
+    size_t sa, sb;            // scales
+    size_t sa_term, sb_term;  // bytes of scales per term
+    size_t inter_a[FMM_MAX_LEVELS], inter_b[FMM_MAX_LEVELS];  // fp32 combinations of outer levels
+    size_t total;
+};
+
+struct fmm_plan {
+    int rank, levels;
+    fmm_quant_params_t qp;
+    float U[FMM_MAX_RANK][4], V[FMM_MAX_RANK][4], W[FMM_MAX_RANK][4];
+    int terms;
+    int device;
+    // device tables
+    int* d_status;            // [4] status words
+    int* d_out_start;         // [terms + 1]
+    FmmOutEntry* d_out;       // [total entries], block offsets in units of leaf blocks (scaled at launch)
+    int n_out_total;
+    int last_launches;
+};
+
+struct EncodeParams {
+    const float* in;          // batch of matrices, each 2*rows x 2*cols (or rows x cols when nq == 1)
+    int64_t in_batch_stride;  // elements between consecutive input matrices
+    int64_t ld;               // leading dimension of the input matrices
+    int batch;                // number of input matrices
+    int rows, cols;           // leaf (output) dimensions per combination
+    int nq;                   // 4: combine quadrants; 1: plain quantization of the matrix itself
+    int R;                    // combinations per input matrix
+    float coef[FMM_MAX_RANK][4];
+    uint8_t* q_out;           // codes, term t = b * R + r at q_out + t * rows * cols
+    void* s_out;              // scales
+    int64_t s_term_stride;    // bytes
+    float amax_floor;
+};
+
+struct CombParams {
+    const float* in;
+    int64_t in_batch_stride, ld;
+    int batch, rows, cols, R;
+    float coef[FMM_MAX_RANK][4];
+    float* out;               // dense rows x cols per (b, r)
+};
+
+fmm_status_t fmm_launch_comb(const CombParams& p, cudaStream_t st);
+fmm_status_t fmm_launch_encode_a(const EncodeParams& p, int blk, int mode, cudaStream_t st);
+fmm_status_t fmm_launch_encode_b(const EncodeParams& p, int blk, int mode, cudaStream_t st);
+
+struct GemmParams {
+    const uint8_t* qa; const uint8_t* qb;   // terms x m x k, terms x n x k
+    const void* sa; const void* sb;
+    int64_t sa_term, sb_term;               // bytes per term
+    float* C; int64_t ldc;                  // full output
+    int64_t Mfull, Nfull;
+    int m, n, k, terms;
+    const int* out_start; const FmmOutEntry* out;
+    int* status;
+};
+fmm_status_t fmm_launch_gemm(const GemmParams& p, int blk, int mode, cudaStream_t st, int* launches);
+
+static inline int64_t fmm_ipow(int64_t b, int e) { int64_t r = 1; while (e-- > 0) r *= b; return r; }

@@ -1,0 +1,154 @@
+// Error measurement (paper App. E.2: relative Frobenius error against an fp64 product;
+// Eq. (D.9) compares the RMS of that error across realizations).
+//   fmm_ref_gemm_fp64 : Cref = A * B with fp64 multiply-accumulate of the fp32 inputs (DFMA tiles).
+//   fmm_error_stats   : sum (C - Cref)^2, sum Cref^2, max |C - Cref| with fp64 accumulation,
+//                       warp-shuffle + shared-memory tree per block, fixed block partition and a
+//                       single-block second stage, hence bit-reproducible.
+#include "fmm_internal.h"
+
+namespace {
+
+constexpr int STAT_BLOCKS = 1024;
+constexpr int STAT_THREADS = 256;
+
+__device__ __forceinline__ void warp_reduce3(double& a, double& b, double& c)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        a += __shfl_xor_sync(0xffffffffu, a, o);
+        b += __shfl_xor_sync(0xffffffffu, b, o);
+        c = fmax(c, __shfl_xor_sync(0xffffffffu, c, o));
+    }
+}
+
+__device__ __forceinline__ void block_reduce3(double& a, double& b, double& c, double* sm)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    warp_reduce3(a, b, c);
+    if (lane == 0) { sm[warp * 3] = a; sm[warp * 3 + 1] = b; sm[warp * 3 + 2] = c; }
+    __syncthreads();
+    if (warp == 0) {
+        const int nw = blockDim.x >> 5;
+        a = lane < nw ? sm[lane * 3] : 0.0;
+        b = lane < nw ? sm[lane * 3 + 1] : 0.0;
+        c = lane < nw ? sm[lane * 3 + 2] : 0.0;
+        warp_reduce3(a, b, c);
+    }
+}
+
+__global__ void __launch_bounds__(STAT_THREADS) error_partial_kernel(const float* __restrict__ C,
+                                                                    const double* __restrict__ Cref,
+                                                                    int64_t count, double* __restrict__ partial)
+{
+    __shared__ double sm[3 * (STAT_THREADS / 32)];
+    double sd = 0.0, sr = 0.0, mx = 0.0;
+    // each thread takes pairs: one 8-byte load of C, one 16-byte load of Cref (count is even)
+    const int64_t pairs = count >> 1;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < pairs; i += (int64_t)gridDim.x * blockDim.x) {
+        const float2 c = __ldcs(reinterpret_cast<const float2*>(C) + i);
+        const double2 r = __ldcs(reinterpret_cast<const double2*>(Cref) + i);
+        const double d0 = (double)c.x - r.x, d1 = (double)c.y - r.y;
+        sd = fma(d0, d0, sd); sd = fma(d1, d1, sd);
+        sr = fma(r.x, r.x, sr); sr = fma(r.y, r.y, sr);
+        mx = fmax(mx, fmax(fabs(d0), fabs(d1)));
+    }
+    block_reduce3(sd, sr, mx, sm);
+    if (threadIdx.x == 0) {
+        partial[blockIdx.x * 3] = sd; partial[blockIdx.x * 3 + 1] = sr; partial[blockIdx.x * 3 + 2] = mx;
+    }
+}
+
+__global__ void __launch_bounds__(STAT_THREADS) error_final_kernel(const double* __restrict__ partial, int n,
+                                                                  double* __restrict__ out3)
+{
+    __shared__ double sm[3 * (STAT_THREADS / 32)];
+    double sd = 0.0, sr = 0.0, mx = 0.0;
+    for (int i = threadIdx.x; i < n; i += blockDim.x) {
+        sd += partial[i * 3]; sr += partial[i * 3 + 1]; mx = fmax(mx, partial[i * 3 + 2]);
+    }
+    block_reduce3(sd, sr, mx, sm);
+    if (threadIdx.x == 0) { out3[0] = sd; out3[1] = sr; out3[2] = mx; }
+}
+
+// 64x64 output tile per block of 16x16 threads, 4x4 outputs per thread, K step 16.
+__global__ void __launch_bounds__(256) ref_gemm_fp64_kernel(const float* __restrict__ A, const float* __restrict__ B,
+                                                           double* __restrict__ C, int64_t M, int64_t N, int64_t K)
+{
+    __shared__ float As[16][64 + 1];   // [k][m]
+    __shared__ float Bs[16][64];       // [k][n]
+    const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+    const int64_t m0 = (int64_t)blockIdx.y * 64, n0 = (int64_t)blockIdx.x * 64;
+    double acc[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = 0.0;
+    for (int64_t k0 = 0; k0 < K; k0 += 16) {
+        // A tile: 64 rows x 16 k = 1024 floats, 4 per thread
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const int idx = threadIdx.x + e * 256;
+            const int r = idx >> 4, kk = idx & 15;
+            As[kk][r] = A[(m0 + r) * K + k0 + kk];
+        }
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const int idx = threadIdx.x + e * 256;
+            const int kk = idx >> 6, c = idx & 63;
+            Bs[kk][c] = B[(k0 + kk) * N + n0 + c];
+        }
+        __syncthreads();
+#pragma unroll
+        for (int kk = 0; kk < 16; ++kk) {
+            double a[4], b[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) a[i] = (double)As[kk][ty * 4 + i];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) b[j] = (double)Bs[kk][tx * 4 + j];
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) acc[i][j] = fma(a[i], b[j], acc[i][j]);
+        }
+        __syncthreads();
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        double* c = C + (m0 + ty * 4 + i) * N + n0 + tx * 4;
+        reinterpret_cast<double2*>(c)[0] = make_double2(acc[i][0], acc[i][1]);
+        reinterpret_cast<double2*>(c)[1] = make_double2(acc[i][2], acc[i][3]);
+    }
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t fmm_error_stats_scratch_bytes(void) { return sizeof(double) * 3 * STAT_BLOCKS; }
+
+fmm_status_t fmm_error_stats(const float* C, const double* Cref, int64_t M, int64_t N, double* out3,
+                             void* scratch, size_t scratch_bytes, void* stream)
+{
+    if (!C || !Cref || !out3 || !scratch) return FMM_ERR_INVALID_ARG;
+    if (M <= 0 || N <= 0 || ((M * N) & 1)) return FMM_ERR_SHAPE;
+    if (scratch_bytes < fmm_error_stats_scratch_bytes() || ((uintptr_t)scratch & 15)) return FMM_ERR_WORKSPACE;
+    if (((uintptr_t)C & 7) || ((uintptr_t)Cref & 15)) return FMM_ERR_INVALID_ARG;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    double* partial = static_cast<double*>(scratch);
+    error_partial_kernel<<<STAT_BLOCKS, STAT_THREADS, 0, st>>>(C, Cref, M * N, partial);
+    error_final_kernel<<<1, STAT_THREADS, 0, st>>>(partial, STAT_BLOCKS, out3);
+    return cudaGetLastError() == cudaSuccess ? FMM_OK : FMM_ERR_CUDA;
+}
+
+fmm_status_t fmm_ref_gemm_fp64(const float* A, const float* B, double* Cref, int64_t M, int64_t N, int64_t K,
+                               void* stream)
+{
+    if (!A || !B || !Cref) return FMM_ERR_INVALID_ARG;
+    if (M <= 0 || N <= 0 || K <= 0 || (M % 64) || (N % 64) || (K % 16)) return FMM_ERR_SHAPE;
+    if ((uintptr_t)Cref & 15) return FMM_ERR_INVALID_ARG;
+    dim3 grid((unsigned)(N / 64), (unsigned)(M / 64));
+    ref_gemm_fp64_kernel<<<grid, 256, 0, reinterpret_cast<cudaStream_t>(stream)>>>(A, B, Cref, M, N, K);
+    return cudaGetLastError() == cudaSuccess ? FMM_OK : FMM_ERR_CUDA;
+}
+
+}  // extern "C"
