@@ -1,0 +1,349 @@
+#!/usr/bin/env python
+"""Benchmark of the block-scaled e4m3 fast-matmul hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+                    [--n 8192] [--levels 1] [--realization phi_optimal]
+                    [--scale-mode fp32|ue8m0] [--block-k 32|128] [--no-variants]
+
+One "step" is one pass of the whole hot path (fmm_matmul: pre-addition + quantization of both
+operands, the 7^levels block-scaled fp8 products on the tensor cores, fused post-addition) over one
+pair of synthetic N(0,1) fp32 operands.  The metric is effective TFLOP/s = 2*M*N*K / time.
+
+The path does not shard (one GPU per matmul, no exchange step): with --gpus N every rank runs an
+independent replica of the same problem and the value is the sum over ranks ("replicas only").
+
+--impl reference times the CPU oracle (oracle/, test infrastructure) on a bounded sample instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "effective fp8 TFLOP/s (2*M*N*K/t), one-level rank-7 block-scaled e4m3 matmul, n=8192"
+UNIT = "TFLOP/s"
+
+
+def parse():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--n", type=int, default=8192)
+    ap.add_argument("--levels", type=int, default=1)
+    ap.add_argument("--realization", default="phi_optimal")
+    ap.add_argument("--scale-mode", default="fp32", choices=["fp32", "ue8m0"])
+    ap.add_argument("--block-k", type=int, default=32, choices=[32, 128])
+    ap.add_argument("--no-variants", action="store_true")
+    ap.add_argument("--ref-n", type=int, default=1024, help="sample size of one reference (oracle) step")
+    ap.add_argument("--cpu-baseline-n", type=int, default=0, help="0 = 4096 with >= 8 host threads, else 2048")
+    return ap.parse_args()
+
+
+# ------------------------------------------------------------------------------------------------
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return {"hbm_gbs": float(d["hbm_gbs"]), "bf16_tflops": float(d["bf16_tflops"]),
+                "bf16_tflops_sustained": float(d.get("bf16_tflops_sustained", d["bf16_tflops"])), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.t = threading.Thread(target=self._read, daemon=True)
+            self.t.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=2)
+        except Exception:
+            pass
+        sm, smax, power, reasons = [], [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); smax.append(float(f[2])); power.append(float(f[3]))
+            except ValueError:
+                continue
+            for nm, v in zip(names, f[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(nm)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        busy = sorted(sm)[len(sm) // 2:]          # the loaded half of the samples
+        return {"sm_mhz": statistics.median(busy), "sm_max_mhz": max(smax), "power_w_max": max(power),
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def algorithmic_work(M, N, K, levels, rank, scale_bytes, blk):
+    """Flops of the products and HBM bytes the method itself must move (fused post-addition):
+    read A and B once, write then read the quantized operands and their scales once, write C once."""
+    f = (rank / 8.0) ** levels if levels > 0 else 1.0
+    r = (rank / 4.0) ** levels if levels > 0 else 1.0
+    flops = 2.0 * M * N * K * f
+    qbytes = r * (M * K + K * N) * (1.0 + scale_bytes / blk)
+    enc_bytes = 4.0 * (M * K + K * N) + qbytes
+    gemm_bytes = qbytes + 4.0 * M * N
+    return flops, enc_bytes, gemm_bytes
+
+
+def run_ours(args):
+    import numpy as np
+    import torch
+    from paper_2609_26077_b200 import fmm, realizations as P
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank_id = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device (the hot path has no CPU fallback)")
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    n, K_steps, W_steps = args.n, args.steps, max(args.warmup, 3)
+    M = N = K = n
+    pk = peaks()
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(1234 + rank_id)
+    A = torch.randn(M, K, device="cuda", generator=gen)
+    B = torch.randn(K, N, device="cuda", generator=gen)
+    C = torch.empty(M, N, device="cuda")
+
+    def make_plan(name, levels, blk, mode):
+        if name == "cubic" or levels == 0:
+            return fmm.Plan(levels=0, block_k=blk, scale_mode=mode)
+        return fmm.Plan(*P.get(name), levels=levels, block_k=blk, scale_mode=mode)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def time_steps(fn, steps, warm):
+        for _ in range(warm):
+            fn()
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            fn()
+        e1.record()
+        barrier()
+        ms = e0.elapsed_time(e1)
+        if dist is not None:
+            t = torch.tensor([ms], device="cuda", dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms / steps
+
+    plan = make_plan(args.realization, args.levels, args.block_k, args.scale_mode)
+    ws = plan.workspace(M, N, K)
+    sampler = ClockSampler(local)
+
+    # ---- timed region 1: K steps of the public call, inputs resident in HBM
+    sampler.start()
+    ms_step = time_steps(lambda: plan.matmul(A, B, out=C, workspace=ws), K_steps, W_steps)
+    launches_per_step = plan.last_launch_count()
+
+    # ---- timed region 2: the same K steps with the two phases bracketed by events (roofline of the dominant kernel)
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(K_steps)]
+    barrier()
+    for i in range(K_steps):
+        ev[i][0].record()
+        plan.encode_only(A, B, workspace=ws)
+        ev[i][1].record()
+        plan.multiply_only(M, N, K, C, workspace=ws)
+        ev[i][2].record()
+    barrier()
+    enc_ms = statistics.mean(e[0].elapsed_time(e[1]) for e in ev)
+    mul_ms = statistics.mean(e[1].elapsed_time(e[2]) for e in ev)
+    clocks = sampler.stop()
+    status = plan.device_status()
+
+    # ---- end to end: host buffers, copies inside the timed region
+    Ah = torch.empty(M, K, dtype=torch.float32, pin_memory=True)
+    Bh = torch.empty(K, N, dtype=torch.float32, pin_memory=True)
+    Ch = torch.empty(M, N, dtype=torch.float32, pin_memory=True)
+    Ah.copy_(A); Bh.copy_(B)
+    Ad, Bd = torch.empty_like(A), torch.empty_like(B)
+
+    def e2e_step():
+        Ad.copy_(Ah, non_blocking=True)
+        Bd.copy_(Bh, non_blocking=True)
+        plan.matmul(Ad, Bd, out=C, workspace=ws)
+        Ch.copy_(C, non_blocking=True)
+
+    e2e_steps = max(3, min(K_steps, 10))
+    ms_e2e = time_steps(e2e_step, e2e_steps, 3)
+
+    flop_eff = 2.0 * M * N * K
+    value = world * flop_eff / (ms_step * 1e-3) / 1e12
+    scale_bytes = 4 if args.scale_mode == "fp32" else 1
+    rank_r = plan.rank if args.levels > 0 else 8
+    flops_alg, enc_bytes, gemm_bytes = algorithmic_work(M, N, K, args.levels, rank_r, scale_bytes, args.block_k)
+    fp8_peak = 2.0 * pk["bf16_tflops"]           # nominal fp8 : bf16 ratio applied to the measured bf16 burst
+    hbm = pk["hbm_gbs"]
+
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K_steps, "warmup": W_steps,
+        "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "fp8_e4m3", "data": "synthetic",
+        "config": {"workload": f"n={n} square, {args.levels} level(s), {args.realization}, A,B iid N(0,1) fp32 (BASELINE configs[2])",
+                   "scale_mode": args.scale_mode, "block_k": args.block_k, "M": M, "N": N, "K": K,
+                   "l2": "inputs larger than L2 (2 x 268 MB fp32 operands, 268 MB output)",
+                   "multi_gpu": "replicas only"},
+        "clocks": clocks,
+        "gpu_launches": launches_per_step * K_steps,
+        "e2e": {"value": world * flop_eff / (ms_e2e * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": ms_e2e,
+                "h2d_bytes_per_step": 4 * (M * K + K * N), "d2h_bytes_per_step": 4 * M * N, "steps": e2e_steps},
+        "phases": {"encode_ms": enc_ms, "multiply_ms": mul_ms,
+                   "encode_hbm_frac": enc_bytes / (enc_ms * 1e-3) / 1e9 / hbm,
+                   "encode_gbs": enc_bytes / (enc_ms * 1e-3) / 1e9,
+                   "multiply_tflops": flops_alg / (mul_ms * 1e-3) / 1e12},
+        "device_status": status[1],
+    }
+    # dominant kernel = the tcgen05 product kernel
+    t_roof_ms = (flops_alg / (fp8_peak * 1e12) + (enc_bytes + gemm_bytes) / (hbm * 1e9)) * 1e3
+    out["roofline"] = {"kernel": "fmm_gemm_kernel", "bound": "tensor",
+                       "achieved": flops_alg / (mul_ms * 1e-3) / 1e12, "peak": fp8_peak, "unit": "TFLOP/s",
+                       "frac": flops_alg / (mul_ms * 1e-3) / 1e12 / fp8_peak, "traffic": None,
+                       "peak_source": f"2 x {pk['source']} bf16 burst ({pk['bf16_tflops']} TF/s)",
+                       "combined_roofline_ms": t_roof_ms, "combined_frac": t_roof_ms / ms_step}
+    if args.scale_mode == "fp32":
+        # the per-block fp32 x fp32 scale promotion runs on the CUDA cores: M*N*(K/blk) x (1 mul + 1 fma) lane-ops
+        f = (rank_r / 8.0) ** args.levels if args.levels > 0 else 1.0
+        lane_ops = 2.0 * M * N * (K / args.block_k) * f
+        alu_peak = 148 * 128 * 1.965e9              # fp32 lanes x max SM clock, one op per lane per clock
+        out["roofline"].update({"bound": "alu" if lane_ops / alu_peak > flops_alg / (fp8_peak * 1e12) else "tensor",
+                                "alu_lane_ops": lane_ops, "alu_peak_lane_ops_per_s": alu_peak,
+                                "alu_frac": lane_ops / (mul_ms * 1e-3) / alu_peak})
+
+    if rank_id == 0 and world == 1 and not args.no_variants:
+        variants = []
+        todo = [("cubic", 0, args.block_k, args.scale_mode), ("strassen", 1, args.block_k, args.scale_mode),
+                ("phi_optimal", 1, 32, "ue8m0"), ("cubic", 0, 32, "ue8m0"),
+                ("phi_optimal", 1, 128, "fp32"), ("cubic", 0, 128, "fp32"), ("phi_optimal", 1, 32, "fp32"),
+                ("phi_optimal", 2, 32, "ue8m0")]
+        seen = {(args.realization, args.levels, args.block_k, args.scale_mode)}
+        for name, lv, blk, mode in todo:
+            if (name, lv, blk, mode) in seen:
+                continue
+            seen.add((name, lv, blk, mode))
+            p2 = make_plan(name, lv, blk, mode)
+            w2 = p2.workspace(M, N, K)
+            ms = time_steps(lambda: p2.matmul(A, B, out=C, workspace=w2), 5, 3)
+            variants.append({"realization": name, "levels": lv, "block_k": blk, "scale_mode": mode,
+                             "ms_per_step": ms, "value": flop_eff / (ms * 1e-3) / 1e12})
+            p2.close()
+        out["variants"] = variants
+        # RMS relative error vs the fp64 product, and ratios vs cubic fp8 in the same quantizer
+        ref = fmm.fmm_ref_gemm_fp64(A, B)
+        errs = {}
+        for name, lv in [("cubic", 0), ("strassen", 1), ("winograd", 1), ("phi_optimal", 1)]:
+            p2 = make_plan(name, lv, args.block_k, args.scale_mode)
+            errs[name] = fmm.rel_frobenius(p2.matmul(A, B, out=C, workspace=p2.workspace(M, N, K)), ref)
+            p2.close()
+        out["error"] = {"rel_frobenius": errs, "ratio_vs_cubic": {k: v / errs["cubic"] for k, v in errs.items()},
+                        "predicted_sqrt_phi_over_8": {"strassen": 2.0, "winograd": 7 ** 0.5, "phi_optimal": 5 / 3}}
+        from oracle import oracle as _O
+        out["cpu_baseline"] = cpu_baseline(args, args.cpu_baseline_n or (4096 if _O.num_threads() >= 8 else 2048))
+    elif rank_id == 0:
+        out["cpu_baseline"] = None
+
+    if rank_id == 0:
+        print(json.dumps(out), flush=True)
+    plan.close()
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+# ------------------------------------------------------------------------------------------------
+def _oracle_step(n, levels, realization, blk, mode, seed=0):
+    import numpy as np
+    from oracle import oracle as O, realizations as R
+    from paper_2609_26077_b200 import workloads as Wl
+    A, B = Wl.gaussian(n, n, n, seed)
+    key = {"phi_optimal": "phi_optimal", "strassen": "strassen", "winograd": "winograd", "cubic": "cubic"}[realization]
+    U, V, W = [np.array(R.to_float(x), dtype=np.float32) for x in R.NAMED[key]()]
+    t0 = time.perf_counter()
+    O.fused_fmm(A, B, U, V, W, levels=levels, blk=blk, mode=O.SCALE_FP32 if mode == "fp32" else O.SCALE_UE8M0)
+    return time.perf_counter() - t0
+
+
+def cpu_baseline(args, n):
+    from oracle import oracle as O
+    t = _oracle_step(n, args.levels, args.realization, args.block_k, args.scale_mode)
+    return {"value": 2.0 * n ** 3 / t / 1e12, "unit": UNIT, "cores": O.num_threads(), "kind": "oracle",
+            "seconds": t, "sample": f"one oracle pass of the same path at n={n} (same realization, levels, quantizer), "
+                                    f"scaled by 2n^3/t; the full n={args.n} case costs (n/{n})^3 more"}
+
+
+def run_reference(args):
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    from oracle import oracle as O
+    n = args.ref_n
+    for _ in range(args.warmup):
+        _oracle_step(n, args.levels, args.realization, args.block_k, args.scale_mode)
+    ts = [_oracle_step(n, args.levels, args.realization, args.block_k, args.scale_mode, seed=i)
+          for i in range(args.steps)]
+    t = sum(ts) / len(ts)
+    val = 2.0 * n ** 3 / t / 1e12
+    sample = f"each step = one oracle pass at n={n} (bounded sample of the n={args.n} workload), value = 2n^3/t"
+    out = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
+           "steps": args.steps, "warmup": args.warmup, "ms_per_step": t * 1e3, "higher_is_better": True,
+           "scaling": "weak", "vs_baseline": None, "dtype": "fp8_e4m3", "data": "synthetic",
+           "config": {"workload": f"n={args.n} square, {args.levels} level(s), {args.realization}, A,B iid N(0,1) fp32 (BASELINE configs[2])",
+                      "scale_mode": args.scale_mode, "block_k": args.block_k, "sample_n": n},
+           "cpu_baseline": {"value": val, "unit": UNIT, "cores": O.num_threads(), "kind": "oracle", "sample": sample},
+           "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+           "gpu_launches": 0}
+    print(json.dumps(out), flush=True)
+
+
+if __name__ == "__main__":
+    a = parse()
+    if a.impl == "reference":
+        run_reference(a)
+    else:
+        run_ours(a)
