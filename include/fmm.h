@@ -115,7 +115,7 @@ fmm_status_t fmm_multiply_only(const fmm_plan_t* plan, float* C, int64_t M, int6
  *   FP32 scale mode: fp32 scales; side 'A': scale_rows x scale_cols = (M/d) x (K/d/block_k) row-major;
  *             side 'B': (K/d/block_k) x (N/d) row-major.
  *   UE8M0 mode: one biased-exponent byte per block in 512-byte tiles of 128 rows x 4 blocks:
- *             tile index (row/128) * (nblocks/4) + (block/4), byte (row%32)*16 + ((row%128)/32)*4 + block%4
+ *             tile index (block/4) * (rows/128) + (row/128), byte (row%32)*16 + ((row%128)/32)*4 + block%4
  *             where row is the M/d (side 'A') or N/d (side 'B') index; scale_rows x scale_cols then
  *             report that logical (rows x blocks) shape. */
 fmm_status_t fmm_quantized_view(const fmm_plan_t* plan, int64_t M, int64_t N, int64_t K, int term,

@@ -259,10 +259,10 @@ fmm_status_t fmm_plan_create(fmm_plan_t** out, int rank, const float* U, const f
     start[p->terms] = (int)entries.size();
     p->n_out_total = (int)entries.size();
 
-    cudaError_t ce = cudaMalloc(&p->d_status, 4 * sizeof(int));
+    cudaError_t ce = cudaMalloc(&p->d_status, 64 * sizeof(int));
     if (ce == cudaSuccess) ce = cudaMalloc(&p->d_out_start, sizeof(int) * start.size());
     if (ce == cudaSuccess) ce = cudaMalloc(&p->d_out, sizeof(FmmOutEntry) * (entries.size() + 1));
-    if (ce == cudaSuccess) ce = cudaMemset(p->d_status, 0, 4 * sizeof(int));
+    if (ce == cudaSuccess) ce = cudaMemset(p->d_status, 0, 64 * sizeof(int));
     if (ce == cudaSuccess) ce = cudaMemcpy(p->d_out_start, start.data(), sizeof(int) * start.size(), cudaMemcpyHostToDevice);
     if (ce == cudaSuccess && !entries.empty())
         ce = cudaMemcpy(p->d_out, entries.data(), sizeof(FmmOutEntry) * entries.size(), cudaMemcpyHostToDevice);
@@ -372,6 +372,14 @@ fmm_status_t fmm_device_status(const fmm_plan_t* plan, int* code)
     *code = h[0];
     return h[0] ? FMM_ERR_DEVICE_TIMEOUT : FMM_OK;
 }
+
+#ifdef FMM_TIMING
+// experiment builds only: raw copy of the status / timing words
+fmm_status_t fmm_debug_status64(const fmm_plan_t* plan, int* out64)
+{
+    return cudaMemcpy(out64, plan->d_status, 64 * sizeof(int), cudaMemcpyDeviceToHost) == cudaSuccess ? FMM_OK : FMM_ERR_CUDA;
+}
+#endif
 
 fmm_status_t fmm_last_launch_count(const fmm_plan_t* plan, int* launches)
 {

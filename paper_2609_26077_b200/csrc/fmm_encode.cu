@@ -11,8 +11,10 @@
 // Both kernels are HBM-bound streaming kernels: every input element is read once with
 // full-line coalesced loads and every output byte is written once in whole 32-byte sectors.
 #include "fmm_internal.h"
+#include "fmm_ptx.cuh"
 
 namespace {
+using fmmptx::pack2; using fmmptx::unpack2; using fmmptx::mul2; using fmmptx::fma2;
 
 __device__ __forceinline__ uint16_t cvt_e4m3x2(float hi, float lo)
 {
@@ -59,12 +61,16 @@ __device__ __forceinline__ float block_scale(float amax, float floor_, float& s_
 
 // ---------------------------------------------------------------------------------------------
 // A side.  One warp handles 128 consecutive k of one output row: 32 lanes x float4, a 512-byte
-// coalesced read per quadrant.  A block of BLK elements is held by BLK/4 adjacent lanes, so the
-// amax is a short butterfly.  Codes leave as one 128-byte store per warp and combination.
+// coalesced read per quadrant.  A block of BLK elements is held by BLK/4 adjacent lanes.  All R
+// combinations are formed first (two elements per fp32x2 instruction); their R block maxima are
+// reduced with a transposing butterfly that leaves combination (lane & 7) in each lane, so the
+// two IEEE divisions of a block are executed once per block instead of once per lane and
+// combination; the multiplier is then broadcast back with one shuffle per combination.
 template <int BLK, int MODE>
 __global__ void __launch_bounds__(256) encode_a_kernel(const EncodeParams p)
 {
     constexpr int GROUP = BLK / 4;                 // lanes per block
+    constexpr unsigned FULL = 0xffffffffu;
     const int lane = threadIdx.x & 31;
     const int64_t warp_gid = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
@@ -73,6 +79,8 @@ __global__ void __launch_bounds__(256) encode_a_kernel(const EncodeParams p)
     const int64_t units = (int64_t)p.batch * p.rows * chunks;
     const int64_t qoff[4] = {0, (int64_t)p.cols, (int64_t)p.rows * p.ld, (int64_t)p.rows * p.ld + p.cols};
     const int64_t term_codes = (int64_t)p.rows * p.cols;
+    const bool b2 = lane & 4, b1 = lane & 2, b0 = lane & 1;
+    const int my_r = lane & 7;
 
     for (int64_t u = warp_gid; u < units; u += nwarps) {
         const int c = (int)(u % chunks);
@@ -80,51 +88,85 @@ __global__ void __launch_bounds__(256) encode_a_kernel(const EncodeParams p)
         const int i = (int)(bi % p.rows);
         const int b = (int)(bi / p.rows);
         const float* base = p.in + (int64_t)b * p.in_batch_stride + (int64_t)i * p.ld + c * 128 + lane * 4;
-        float4 x[4];
+        unsigned long long xl[4], xh[4];
 #pragma unroll
         for (int j = 0; j < 4; ++j)
-            if (j < p.nq) x[j] = __ldcs(reinterpret_cast<const float4*>(base + qoff[j]));
+            if (j < p.nq) {
+                const float4 x = __ldcs(reinterpret_cast<const float4*>(base + qoff[j]));
+                xl[j] = pack2(x.x, x.y); xh[j] = pack2(x.z, x.w);
+            }
 
-        for (int r = 0; r < p.R; ++r) {
-            float v0 = 0.f, v1 = 0.f, v2 = 0.f, v3 = 0.f;
-            bool set = false;
+        unsigned long long vl[FMM_MAX_RANK], vh[FMM_MAX_RANK];
+        float am[FMM_MAX_RANK];
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                const float cj = p.coef[r][j];
-                if (cj != 0.0f) {
-                    if (!set) {
-                        v0 = __fmul_rn(cj, x[j].x); v1 = __fmul_rn(cj, x[j].y);
-                        v2 = __fmul_rn(cj, x[j].z); v3 = __fmul_rn(cj, x[j].w);
-                        set = true;
-                    } else {
-                        v0 = __fmaf_rn(cj, x[j].x, v0); v1 = __fmaf_rn(cj, x[j].y, v1);
-                        v2 = __fmaf_rn(cj, x[j].z, v2); v3 = __fmaf_rn(cj, x[j].w, v3);
+        for (int r = 0; r < FMM_MAX_RANK; ++r) {
+            vl[r] = 0ull; vh[r] = 0ull; am[r] = 0.0f;
+            if (r < p.R) {
+                bool set = false;
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const float cj = p.coef[r][j];
+                    if (cj != 0.0f) {
+                        const unsigned long long c2 = pack2(cj, cj);
+                        if (!set) { vl[r] = mul2(c2, xl[j]); vh[r] = mul2(c2, xh[j]); set = true; }
+                        else { vl[r] = fma2(c2, xl[j], vl[r]); vh[r] = fma2(c2, xh[j], vh[r]); }
                     }
                 }
+                float a0, a1, a2, a3;
+                unpack2(vl[r], a0, a1); unpack2(vh[r], a2, a3);
+                am[r] = fmaxf(fmaxf(fabsf(a0), fabsf(a1)), fmaxf(fabsf(a2), fabsf(a3)));
             }
-            float amax = fmaxf(fmaxf(fabsf(v0), fabsf(v1)), fmaxf(fabsf(v2), fabsf(v3)));
+        }
+        // transposing butterfly over the 8 lanes (lane & 7): afterwards `mine` is the maximum of
+        // combination (lane & 7) over those lanes
+        float w[4], x2[2], mine;
 #pragma unroll
-            for (int o = 1; o < GROUP; o <<= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
-            float s; uint32_t e8;
-            const float inv = block_scale<MODE>(amax, p.amax_floor, s, e8);
-            const uint32_t packed = pack4_e4m3(__fmul_rn(v0, inv), __fmul_rn(v1, inv),
-                                               __fmul_rn(v2, inv), __fmul_rn(v3, inv));
-            const int64_t t = (int64_t)b * p.R + r;
-            *reinterpret_cast<uint32_t*>(p.q_out + t * term_codes + (int64_t)i * p.cols + c * 128 + lane * 4) = packed;
-            if (MODE == FMM_SCALE_FP32_AMAX_DIV_448) {
-                if ((lane % GROUP) == 0) {
-                    float* so = reinterpret_cast<float*>(reinterpret_cast<char*>(p.s_out) + t * p.s_term_stride);
-                    so[(int64_t)i * nkb + c * (128 / BLK) + lane / GROUP] = s;
-                }
-            } else {
-                // four exponent bytes of this row (blocks 4c .. 4c+3) form one aligned word of the scale tile
-                uint32_t w = __shfl_sync(0xffffffffu, e8, 0) | (__shfl_sync(0xffffffffu, e8, 8) << 8) |
-                             (__shfl_sync(0xffffffffu, e8, 16) << 16) | (__shfl_sync(0xffffffffu, e8, 24) << 24);
-                if (lane == 0) {
-                    char* so = reinterpret_cast<char*>(p.s_out) + t * p.s_term_stride;
-                    const int64_t tile = (int64_t)(i >> 7) * (nkb >> 2) + c;
-                    *reinterpret_cast<uint32_t*>(so + tile * 512 + (i & 31) * 16 + ((i & 127) >> 5) * 4) = w;
-                }
+        for (int j = 0; j < 4; ++j) {
+            const float send = b2 ? am[j] : am[j + 4], keep = b2 ? am[j + 4] : am[j];
+            w[j] = fmaxf(keep, __shfl_xor_sync(FULL, send, 4));
+        }
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+            const float send = b1 ? w[j] : w[j + 2], keep = b1 ? w[j + 2] : w[j];
+            x2[j] = fmaxf(keep, __shfl_xor_sync(FULL, send, 2));
+        }
+        {
+            const float send = b0 ? x2[0] : x2[1], keep = b0 ? x2[1] : x2[0];
+            mine = fmaxf(keep, __shfl_xor_sync(FULL, send, 1));
+        }
+        if (GROUP == 32) {
+            mine = fmaxf(mine, __shfl_xor_sync(FULL, mine, 8));
+            mine = fmaxf(mine, __shfl_xor_sync(FULL, mine, 16));
+        }
+        float s; uint32_t e8;
+        const float inv = block_scale<MODE>(mine, p.amax_floor, s, e8);
+
+        uint8_t* qrow = p.q_out + ((int64_t)b * p.R) * term_codes + (int64_t)i * p.cols + c * 128 + lane * 4;
+#pragma unroll
+        for (int r = 0; r < FMM_MAX_RANK; ++r) {
+            if (r < p.R) {
+                const float inv_r = __shfl_sync(FULL, inv, (GROUP == 32) ? r : ((lane & 24) | r));
+                const unsigned long long i2 = pack2(inv_r, inv_r);
+                float y0, y1, y2, y3;
+                unpack2(mul2(vl[r], i2), y0, y1); unpack2(mul2(vh[r], i2), y2, y3);
+                *reinterpret_cast<uint32_t*>(qrow + r * term_codes) = pack4_e4m3(y0, y1, y2, y3);
+            }
+        }
+        // scales: lane holds the scale of combination my_r, block (lane / GROUP) of this chunk
+        if (MODE == FMM_SCALE_FP32_AMAX_DIV_448) {
+            if (my_r < p.R && (GROUP == 8 || lane < 8)) {
+                float* so = reinterpret_cast<float*>(reinterpret_cast<char*>(p.s_out) + ((int64_t)b * p.R + my_r) * p.s_term_stride);
+                so[(int64_t)i * nkb + c * (128 / BLK) + (GROUP == 8 ? (lane >> 3) : 0)] = s;
+            }
+        } else {
+            // four exponent bytes of this row (blocks 4c .. 4c+3) form one aligned word of the scale tile
+            uint32_t wv = e8 << (8 * (lane >> 3));
+            wv |= __shfl_xor_sync(FULL, wv, 8);
+            wv |= __shfl_xor_sync(FULL, wv, 16);
+            if (lane < 8 && lane < p.R) {
+                char* so = reinterpret_cast<char*>(p.s_out) + ((int64_t)b * p.R + lane) * p.s_term_stride;
+                const int64_t tile = (int64_t)c * (p.rows >> 7) + (i >> 7);
+                *reinterpret_cast<uint32_t*>(so + tile * 512 + (i & 31) * 16 + ((i & 127) >> 5) * 4) = wv;
             }
         }
     }
@@ -132,85 +174,91 @@ __global__ void __launch_bounds__(256) encode_a_kernel(const EncodeParams p)
 
 // ---------------------------------------------------------------------------------------------
 // B side.  Blocks run along k, the strided axis of row-major B, and the output is K-major (the
-// tensor-core operand layout).  One thread owns one column n: each of its loads is part of a
-// 128-byte coalesced warp read of a B row; the amax is thread-local; the 32 codes of a block
-// leave as 32 contiguous bytes.  BLK == 128 takes a second pass over the four 32-element
-// sub-blocks (served by L1/L2) because the whole block does not fit in registers.
+// tensor-core operand layout).  A thread owns 16 consecutive k of one column n; lanes l and l+16
+// hold the two halves of a 32-element (sub-)block, so one shuffle completes the amax.  Each load
+// is two 64-byte row segments per warp; each thread writes 16 contiguous code bytes and the two
+// lanes of a block fill one 32-byte sector.  BLK == 128 takes a second pass over the four
+// 32-element sub-blocks (served by L1/L2).
 template <int MODE>
-__device__ __forceinline__ void store_b_scale(const EncodeParams& p, int64_t t, int j, int kb, int nkb,
+__device__ __forceinline__ void store_b_scale(const EncodeParams& p, int64_t t, int j, int kb, int kc,
                                               float s, uint32_t e8word, bool last_of_word)
 {
     char* so = reinterpret_cast<char*>(p.s_out) + t * p.s_term_stride;
     if (MODE == FMM_SCALE_FP32_AMAX_DIV_448) {
         reinterpret_cast<float*>(so)[(int64_t)kb * p.cols + j] = s;
     } else if (last_of_word) {
-        const int64_t tile = (int64_t)(j >> 7) * (nkb >> 2) + (kb >> 2);
+        const int64_t tile = (int64_t)kc * (p.cols >> 7) + (j >> 7);
         *reinterpret_cast<uint32_t*>(so + tile * 512 + (j & 31) * 16 + ((j & 127) >> 5) * 4) = e8word;
     }
 }
 
 template <int BLK, int MODE>
-__global__ void __launch_bounds__(128) encode_b_kernel(const EncodeParams p)
+__global__ void __launch_bounds__(128, 4) encode_b_kernel(const EncodeParams p)
 {
     // here p.rows = leaf k (contracted), p.cols = leaf n
-    const int j = blockIdx.x * 128 + threadIdx.x;
+    constexpr unsigned FULL = 0xffffffffu;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int j = blockIdx.x * 64 + warp * 16 + (lane & 15);
+    const int khalf = lane >> 4;
     const int kc = blockIdx.y;                      // chunk of 128 k
     const int b = blockIdx.z;
-    const int nkb = p.rows / BLK;
     const int64_t qoff[4] = {0, (int64_t)p.cols, (int64_t)p.rows * p.ld, (int64_t)p.rows * p.ld + p.cols};
     const float* base = p.in + (int64_t)b * p.in_batch_stride + j;
     const int64_t term_codes = (int64_t)p.rows * p.cols;
 
-    float raw[4][32];
-    float blk_amax[FMM_MAX_RANK];
-    float blk_inv[FMM_MAX_RANK];
-#pragma unroll
-    for (int r = 0; r < FMM_MAX_RANK; ++r) { blk_amax[r] = 0.0f; blk_inv[r] = 0.0f; }
+    float raw[4][16];
+    float blk_amax[FMM_MAX_RANK], blk_inv[FMM_MAX_RANK];
     uint32_t e8word[FMM_MAX_RANK];
 #pragma unroll
-    for (int r = 0; r < FMM_MAX_RANK; ++r) e8word[r] = 0;
+    for (int r = 0; r < FMM_MAX_RANK; ++r) { blk_amax[r] = 0.0f; blk_inv[r] = 0.0f; e8word[r] = 0; }
 
     constexpr int PASSES = (BLK == 32) ? 1 : 2;
 #pragma unroll 1
     for (int pass = 0; pass < PASSES; ++pass) {
 #pragma unroll 1
         for (int sub = 0; sub < 4; ++sub) {
-            const int k0 = kc * 128 + sub * 32;
+            const int k0 = kc * 128 + sub * 32 + khalf * 16;
 #pragma unroll
             for (int jq = 0; jq < 4; ++jq)
                 if (jq < p.nq) {
 #pragma unroll
-                    for (int kk = 0; kk < 32; ++kk)
+                    for (int kk = 0; kk < 16; ++kk)
                         raw[jq][kk] = __ldg(base + qoff[jq] + (int64_t)(k0 + kk) * p.ld);
                 }
 #pragma unroll
             for (int r = 0; r < FMM_MAX_RANK; ++r) {
                 if (r < p.R) {
-                    float v[32];
+                    unsigned long long v[8];
                     bool set = false;
 #pragma unroll
                     for (int jq = 0; jq < 4; ++jq) {
                         const float cj = p.coef[r][jq];
                         if (cj != 0.0f) {
+                            const unsigned long long c2 = pack2(cj, cj);
                             if (!set) {
 #pragma unroll
-                                for (int kk = 0; kk < 32; ++kk) v[kk] = __fmul_rn(cj, raw[jq][kk]);
+                                for (int g = 0; g < 8; ++g) v[g] = mul2(c2, pack2(raw[jq][2 * g], raw[jq][2 * g + 1]));
                                 set = true;
                             } else {
 #pragma unroll
-                                for (int kk = 0; kk < 32; ++kk) v[kk] = __fmaf_rn(cj, raw[jq][kk], v[kk]);
+                                for (int g = 0; g < 8; ++g) v[g] = fma2(c2, pack2(raw[jq][2 * g], raw[jq][2 * g + 1]), v[g]);
                             }
                         }
                     }
                     if (!set) {
 #pragma unroll
-                        for (int kk = 0; kk < 32; ++kk) v[kk] = 0.0f;
+                        for (int g = 0; g < 8; ++g) v[g] = 0ull;
                     }
                     const int64_t t = (int64_t)b * p.R + r;
                     if (BLK == 32 || pass == 0) {
                         float amax = 0.0f;
 #pragma unroll
-                        for (int kk = 0; kk < 32; ++kk) amax = fmaxf(amax, fabsf(v[kk]));
+                        for (int g = 0; g < 8; ++g) {
+                            float a0, a1;
+                            unpack2(v[g], a0, a1);
+                            amax = fmaxf(amax, fmaxf(fabsf(a0), fabsf(a1)));
+                        }
+                        amax = fmaxf(amax, __shfl_xor_sync(FULL, amax, 16));
                         if (BLK == 32) blk_amax[r] = amax; else blk_amax[r] = fmaxf(blk_amax[r], amax);
                     }
                     if (BLK == 32 || (pass == 0 && sub == 3)) {
@@ -218,18 +266,20 @@ __global__ void __launch_bounds__(128) encode_b_kernel(const EncodeParams p)
                         blk_inv[r] = block_scale<MODE>(blk_amax[r], p.amax_floor, s, e8);
                         const int kb = (BLK == 32) ? (kc * 4 + sub) : kc;
                         e8word[r] |= e8 << (8 * (kb & 3));
-                        store_b_scale<MODE>(p, t, j, kb, nkb, s, e8word[r], (kb & 3) == 3);
+                        if (khalf == 0) store_b_scale<MODE>(p, t, j, kb, kc, s, e8word[r], (kb & 3) == 3);
                     }
                     if (BLK == 32 || pass == 1) {
-                        const float inv = blk_inv[r];
-                        uint32_t w[8];
+                        const unsigned long long i2 = pack2(blk_inv[r], blk_inv[r]);
+                        uint32_t wv[4];
 #pragma unroll
-                        for (int g = 0; g < 8; ++g)
-                            w[g] = pack4_e4m3(__fmul_rn(v[4 * g], inv), __fmul_rn(v[4 * g + 1], inv),
-                                              __fmul_rn(v[4 * g + 2], inv), __fmul_rn(v[4 * g + 3], inv));
-                        uint4* dst = reinterpret_cast<uint4*>(p.q_out + t * term_codes + (int64_t)j * p.rows + k0);
-                        dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
-                        dst[1] = make_uint4(w[4], w[5], w[6], w[7]);
+                        for (int g = 0; g < 4; ++g) {
+                            float y0, y1, y2, y3;
+                            unpack2(mul2(v[2 * g], i2), y0, y1);
+                            unpack2(mul2(v[2 * g + 1], i2), y2, y3);
+                            wv[g] = pack4_e4m3(y0, y1, y2, y3);
+                        }
+                        *reinterpret_cast<uint4*>(p.q_out + t * term_codes + (int64_t)j * p.rows + k0) =
+                            make_uint4(wv[0], wv[1], wv[2], wv[3]);
                     }
                 }
             }
@@ -317,7 +367,7 @@ fmm_status_t fmm_launch_encode_a(const EncodeParams& p, int blk, int mode, cudaS
 
 fmm_status_t fmm_launch_encode_b(const EncodeParams& p, int blk, int mode, cudaStream_t st)
 {
-    dim3 grid((unsigned)(p.cols / 128), (unsigned)(p.rows / 128), (unsigned)p.batch);
+    dim3 grid((unsigned)(p.cols / 64), (unsigned)(p.rows / 128), (unsigned)p.batch);
     if (mode == FMM_SCALE_FP32_AMAX_DIV_448) {
         if (blk == 32) encode_b_kernel<32, FMM_SCALE_FP32_AMAX_DIV_448><<<grid, 128, 0, st>>>(p);
         else encode_b_kernel<128, FMM_SCALE_FP32_AMAX_DIV_448><<<grid, 128, 0, st>>>(p);

@@ -2,13 +2,14 @@
 // c = sum_r <U_r,a><V_r,b> W_r; the products M_r = S_r^ * T_r^ of the quantized combinations are
 // accumulated in fp32 and carried into the output blocks by the decoder W_r).
 //
-// One persistent CTA per SM owns an output tile POSITION (the same 128 x BN tile in every output
-// block of C) and walks all terms for it, so the W-weighted accumulation into C is race-free and
-// deterministic without atomics between CTAs.
+// A persistent CTA (NCTA == 1) or CTA pair on two adjacent SMs (NCTA == 2, tcgen05 cta_group::2)
+// owns an output tile POSITION - the same (NCTA*128) x BN tile in every output block of C - and
+// walks all terms for it, so the W-weighted accumulation into C is race-free and deterministic.
 //
-//   warp 0      TMA producer: K-major e4m3 tiles of S_r and T_r (128-byte swizzle) + their scales
-//   warp 1      tcgen05.mma issuer, fp32 accumulators in TMEM
-//   warps 2..9  epilogue: TMEM -> registers -> (x W[r][q]) -> swizzled smem -> TMA store / TMA
+//   warp 0      TMA producer: K-major e4m3 tiles of S_r and T_r (128-byte swizzle) + their scales.
+//               In a pair each CTA loads its own 128 rows of S_r and its own half of the T_r tile.
+//   warp 1      tcgen05.mma issuer (the even CTA of a pair issues for both), fp32 accumulators in TMEM
+//   warps 4..11 epilogue (two warpgroups, given most of the register file with setmaxnreg): TMEM -> registers -> (x W[r][q]) -> swizzled smem -> TMA store / TMA
 //               add-reduce into the C blocks (the read-modify-write happens in L2, not in the SM)
 //
 // Scale handling:
@@ -17,32 +18,50 @@
 //   FP32 mode   (the paper's scale = amax/448 in fp32 on BOTH sides, per 1 x blk block): no
 //               tensor-core path can apply a per-row x per-column fp32 factor per K block, so
 //               each K block's partial product is accumulated on its own in TMEM
-//               (kind::f8f6f4) and promoted on the CUDA cores: acc += P * (sA[row] * sB[col]).
+//               (kind::f8f6f4) and promoted on the CUDA cores: acc += P * (sA[row] * sB[col]),
+//               two columns per instruction (fp32x2), overlapped with the next TMEM load.
 //
 // Every wait is bounded: on time-out a status word is set and all roles leave the kernel.
-#include <stdio.h>
+#include <string.h>
 #include "fmm_internal.h"
+#include "fmm_ptx.cuh"
 
 namespace {
+using namespace fmmptx;
 
-constexpr int BM = 128;
+constexpr int BM = 128;                 // rows per CTA
 constexpr int BK = 128;                 // K elements (= bytes) per pipeline stage: one swizzle row
-constexpr int EPI_WARPS = 8;
-constexpr int NUM_THREADS = (2 + EPI_WARPS) * 32;
+constexpr int EPI_WARPS = 8;               // two per TMEM lane quadrant, each half of the tile's columns
+constexpr int EPI_WARP0 = 4;               // warps 0..3: producer, MMA issuer, two idle (one warpgroup)
+constexpr int NUM_THREADS = (EPI_WARP0 + EPI_WARPS) * 32;
+// setmaxnreg budget: the CTA's register pool is NUM_THREADS x (registers at launch); an increase
+// beyond what the decrease freed would block forever, so the split is checked here.
+constexpr int REGS_AT_LAUNCH = 168, REGS_CTRL = 56, REGS_EPI = 224;
+static_assert(EPI_WARP0 * 32 * REGS_CTRL + EPI_WARPS * 32 * REGS_EPI <= NUM_THREADS * REGS_AT_LAUNCH, "register pool");
+static_assert(NUM_THREADS * (REGS_AT_LAUNCH + 8) > 65536, "REGS_AT_LAUNCH must be the launch-bound maximum");
 constexpr int STAGING_BYTES = 32 * 128; // 32 rows x 32 fp32 per epilogue warp and buffer
-constexpr int STAGING_BUFS = 2;
+#ifndef FMM_EXP_STAGING_BUFS
+#define FMM_EXP_STAGING_BUFS 2
+#endif
+constexpr int STAGING_BUFS = FMM_EXP_STAGING_BUFS;
 
-template <int BN, int MODE, int BLK>
+template <int BN, int MODE, int BLK, int NCTA>
 struct Cfg {
     static constexpr bool MX = (MODE == FMM_SCALE_UE8M0_CEIL);
-    static constexpr int STAGES = (BN == 256) ? 3 : 4;
+    static constexpr int BROWS = BN / NCTA;                  // T_r rows this CTA loads per stage
     static constexpr int A_BYTES = BM * BK;
-    static constexpr int B_BYTES = BN * BK;
-    static constexpr int SF_STAGE_BYTES = MX ? (512 + (BN / 128) * 512) : 0;
+    static constexpr int B_BYTES = BROWS * BK;
+#ifdef FMM_EXP_STAGES
+    static constexpr int STAGES = (NCTA == 2) ? FMM_EXP_STAGES : ((A_BYTES + B_BYTES) > 40000 ? 3 : 4);
+#else
+    static constexpr int STAGES = (A_BYTES + B_BYTES) > 40000 ? 3 : 4;
+#endif
+    static constexpr int SFB_ATOMS = BN / 128;
+    static constexpr int SF_STAGE_BYTES = MX ? (512 + SFB_ATOMS * 512) : 0;
     static constexpr int KB_PER_STAGE = BK / BLK;
     static constexpr int SB_STAGES = STAGES + 1;
     static constexpr int SB_STAGE_BYTES = MX ? 0 : KB_PER_STAGE * BN * 4;
-    static constexpr int TX_BYTES = A_BYTES + B_BYTES + SF_STAGE_BYTES;
+    static constexpr int TX_BYTES = NCTA * (A_BYTES + B_BYTES + SF_STAGE_BYTES);
     static constexpr int OFF_A = 0;
     static constexpr int OFF_B = OFF_A + STAGES * A_BYTES;
     static constexpr int OFF_STG = OFF_B + STAGES * B_BYTES;
@@ -54,100 +73,19 @@ struct Cfg {
     // TMEM: MX: one BN-column accumulator, then per stage 4 SFA + 4*(BN/128) SFB columns.
     //       FP32: ring of 512/BN accumulators, one per K block in flight.
     static constexpr int ACC_BUFS = MX ? 1 : (512 / BN);
-    static constexpr int SF_COLS = 4 + 4 * (BN / 128);
+    static constexpr int SF_COLS = 4 + 4 * SFB_ATOMS;
     static constexpr int CW = BN / 2;      // columns per epilogue warp
     static_assert(SMEM_BYTES <= 232448, "shared memory budget");
     static_assert(!MX || BN + STAGES * SF_COLS <= 512, "TMEM budget");
 };
 
-// ------------------------------------------------------------------------------- PTX wrappers
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
-{ asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count)); }
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
-{ asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory"); }
-__device__ __forceinline__ void mbar_arrive(uint32_t bar)
-{ asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory"); }
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
-{
-    uint32_t ok;
-    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok != 0;
-}
-__device__ __forceinline__ uint64_t global_timer()
-{ uint64_t t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
-
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm, int x, int y, uint32_t bar)
-{
-    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-                 ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tm)), "r"(bar), "r"(x), "r"(y) : "memory");
-}
-__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar)
-{
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(dst), "l"(reinterpret_cast<uint64_t>(src)), "r"(bytes), "r"(bar) : "memory");
-}
-__device__ __forceinline__ void tma_store_2d(const CUtensorMap* tm, int x, int y, uint32_t src)
-{
-    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
-                 ::"l"(reinterpret_cast<uint64_t>(tm)), "r"(src), "r"(x), "r"(y) : "memory");
-}
-__device__ __forceinline__ void tma_reduce_add_2d(const CUtensorMap* tm, int x, int y, uint32_t src)
-{
-    asm volatile("cp.reduce.async.bulk.tensor.2d.global.shared::cta.add.bulk_group [%0, {%2, %3}], [%1];"
-                 ::"l"(reinterpret_cast<uint64_t>(tm)), "r"(src), "r"(x), "r"(y) : "memory");
-}
-__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
-template <int N> __device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
-template <int N> __device__ __forceinline__ void bulk_wait() { asm volatile("cp.async.bulk.wait_group %0;" ::"n"(N) : "memory"); }
-__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_commit(uint32_t bar)
-{ asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory"); }
-__device__ __forceinline__ void tc_cp_32x128b_warpx4(uint32_t taddr, uint64_t sdesc)
-{ asm volatile("tcgen05.cp.cta_group::1.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(sdesc) : "memory"); }
-__device__ __forceinline__ void mma_f8f6f4(uint32_t d, uint64_t a, uint64_t b, uint32_t idesc, uint32_t accumulate)
-{
-    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-                 "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t}"
-                 ::"r"(d), "l"(a), "l"(b), "r"(idesc), "r"(accumulate) : "memory");
-}
-__device__ __forceinline__ void mma_mxf8(uint32_t d, uint64_t a, uint64_t b, uint32_t idesc, uint32_t accumulate,
-                                         uint32_t tsfa, uint32_t tsfb)
-{
-    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-                 "tcgen05.mma.cta_group::1.kind::mxf8f6f4.block_scale [%0], %1, %2, %3, [%5], [%6], p;\n\t}"
-                 ::"r"(d), "l"(a), "l"(b), "r"(idesc), "r"(accumulate), "r"(tsfa), "r"(tsfb) : "memory");
-}
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float* v)
-{
-    uint32_t* r = reinterpret_cast<uint32_t*>(v);
-    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-                 "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-                 "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-                   "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
-                   "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
-                   "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-                 : "r"(taddr) : "memory");
-}
-__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-
-// K-major operand tile, 128-byte swizzle: rows of 128 bytes, 8-row groups 1024 bytes apart.
-__device__ __forceinline__ uint64_t make_kmajor_sw128_desc(uint32_t saddr)
-{
-    return (uint64_t)((saddr & 0x3FFFF) >> 4) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) |
-           ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
-}
-// Scale-factor chunk for tcgen05.cp 32x128b: 32 rows of 16 bytes, no swizzle, 8-row groups 128 bytes apart.
-__device__ __forceinline__ uint64_t make_sf_desc(uint32_t saddr)
-{
-    return (uint64_t)((saddr & 0x3FFFF) >> 4) | ((uint64_t)(128 >> 4) << 32) | ((uint64_t)1 << 46);
-}
+#ifdef FMM_TIMING
+#define TCLK() clock64()
+#define TADD(slot, t0) do { if (blockIdx.x == 0 && lane == 0) tim[slot] += clock64() - (t0); } while (0)
+#else
+#define TCLK() 0ll
+#define TADD(slot, t0) do { (void)(t0); } while (0)
+#endif
 
 constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;   // 2 s: far beyond any legitimate wait
 
@@ -175,7 +113,6 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const C
     }
     return true;
 }
-
 // Same, with a warp-uniform verdict (the epilogue warps execute .sync.aligned instructions afterwards).
 __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, const Ctl& ctl, int where)
 {
@@ -184,19 +121,20 @@ __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, co
 }
 
 struct KParams {
-    const uint8_t* sa; const uint8_t* sb;   // scale arrays (bytes)
+    const uint8_t* sa; const uint8_t* sb;   // scale arrays (bytes); fp32 mode only
     long long sa_term, sb_term;
     int m, n, k, terms;
     const int* out_start; const FmmOutEntry* out;
     int* status;
 };
 
-template <int BN, int MODE, int BLK>
+template <int BN, int MODE, int BLK, int NCTA>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-                const __grid_constant__ CUtensorMap tmC, const KParams p)
+                const __grid_constant__ CUtensorMap tmC, const __grid_constant__ CUtensorMap tmSFA,
+                const __grid_constant__ CUtensorMap tmSFB, const KParams p)
 {
-    using C = Cfg<BN, MODE, BLK>;
+    using C = Cfg<BN, MODE, BLK, NCTA>;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw_addr = smem_u32(smem_raw);
     const uint32_t base = (raw_addr + 1023u) & ~1023u;
@@ -214,52 +152,70 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     const Ctl ctl{abort_flag, p.status};
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int cta_rank = (NCTA == 2) ? (int)cluster_ctarank() : 0;
+    const bool leader = (cta_rank == 0);
+    const int unit = blockIdx.x / NCTA;            // CTA or CTA pair index
+    const int units = gridDim.x / NCTA;
+#ifdef FMM_TIMING
+    long long tim[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    const long long t_kernel = clock64();
+#endif
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < C::STAGES; ++s) { mbar_init(bar_full(s), 1); mbar_init(bar_empty(s), 1); }
         for (int s = 0; s < C::SB_STAGES; ++s) { mbar_init(bar_sfull(s), 1); mbar_init(bar_sempty(s), EPI_WARPS); }
-        for (int b = 0; b < 4; ++b) { mbar_init(bar_tfull(b), 1); mbar_init(bar_tempty(b), EPI_WARPS); }
+        for (int b = 0; b < 4; ++b) { mbar_init(bar_tfull(b), 1); mbar_init(bar_tempty(b), NCTA * EPI_WARPS); }
         *abort_flag = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        fence_barrier_init();
     }
     if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(512) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        tmem_alloc<NCTA>(smem_u32(tmem_slot), 512);
+        tmem_relinquish<NCTA>();
     }
     tc_fence_before();
     __syncthreads();
+    if (NCTA == 2) cluster_sync();                 // the peer's barriers are initialised before anyone signals them
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
     const int tiles_n = p.n / BN;
-    const int positions = (p.m / BM) * tiles_n;
+    const int positions = (p.m / (BM * NCTA)) * tiles_n;
     const int kstages = p.k / BK;
     const int nkb = p.k / BLK;
+    const int row_blocks_a = p.m / 128, row_blocks_b = p.n / 128;
 
+    if (warp < EPI_WARP0) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(REGS_CTRL));
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
             int stage = 0; uint32_t phase = 0;
             int ss = 0; uint32_t sphase = 0;
             bool ok = true;
-            for (int pos = blockIdx.x; pos < positions && ok; pos += gridDim.x) {
+            for (int pos = unit; pos < positions && ok; pos += units) {
                 const int tm = pos / tiles_n, tn = pos % tiles_n;
+                const int row_blk = tm * NCTA + cta_rank;                 // 128-row block of S_r this CTA owns
                 for (int t = 0; t < p.terms && ok; ++t) {
                     for (int ks = 0; ks < kstages; ++ks) {
+                        const long long tw = TCLK();
                         if (!mbar_wait(bar_empty(stage), phase ^ 1u, ctl, 101)) { ok = false; break; }
-                        mbar_expect_tx(bar_full(stage), C::TX_BYTES);
-                        tma_load_2d(base + C::OFF_A + stage * C::A_BYTES, &tmA, ks * BK, t * p.m + tm * BM, bar_full(stage));
-                        tma_load_2d(base + C::OFF_B + stage * C::B_BYTES, &tmB, ks * BK, t * p.n + tn * BN, bar_full(stage));
+                        TADD(0, tw);
+                        // completion is counted on the even CTA's barrier; only that CTA arms it
+                        const uint32_t fb = (NCTA == 2) ? (bar_full(stage) & PEER_BIT_MASK) : bar_full(stage);
+#ifdef FMM_EXP_NO_TMA
+                        if (leader) mbar_arrive(bar_full(stage));
+                        if (++stage == C::STAGES) { stage = 0; phase ^= 1u; }
+                        continue;
+#endif
+                        if (leader) mbar_expect_tx(bar_full(stage), C::TX_BYTES);
+                        tma_load_2d<NCTA>(base + C::OFF_A + stage * C::A_BYTES, &tmA, ks * BK, t * p.m + row_blk * BM, fb);
+                        tma_load_2d<NCTA>(base + C::OFF_B + stage * C::B_BYTES, &tmB, ks * BK,
+                                          t * p.n + tn * BN + cta_rank * C::BROWS, fb);
                         if (C::MX) {
+                            // scale tiles: 512-byte atoms, ordered [term][k quad][128-row block]
                             const uint32_t sf = base + C::OFF_SF + stage * C::SF_STAGE_BYTES;
-                            const uint8_t* ga = p.sa + (long long)t * p.sa_term + ((long long)tm * (nkb >> 2) + ks) * 512;
-                            bulk_load(sf, ga, 512, bar_full(stage));
-#pragma unroll
-                            for (int h = 0; h < BN / 128; ++h) {
-                                const uint8_t* gb = p.sb + (long long)t * p.sb_term +
-                                                    ((long long)(tn * (BN / 128) + h) * (nkb >> 2) + ks) * 512;
-                                bulk_load(sf + 512 + h * 512, gb, 512, bar_full(stage));
-                            }
+                            tma_load_2d<NCTA>(sf, &tmSFA, 0, (t * (nkb >> 2) + ks) * row_blocks_a + row_blk, fb);
+                            tma_load_2d<NCTA>(sf + 512, &tmSFB, 0, (t * (nkb >> 2) + ks) * row_blocks_b + tn * C::SFB_ATOMS, fb);
                         } else {
                             if (!mbar_wait(bar_sempty(ss), sphase ^ 1u, ctl, 102)) { ok = false; break; }
                             mbar_expect_tx(bar_sfull(ss), C::SB_STAGE_BYTES);
@@ -277,22 +233,27 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             }
         }
     } else if (warp == 1) {
-        // ------------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
+        // ------------------------------------------------------------------ MMA issuer (even CTA only in a pair)
+        if (lane == 0 && leader) {
             int stage = 0; uint32_t phase = 0;
             int buf = 0; uint32_t bphase = 0;
             bool ok = true;
+            constexpr uint32_t MDIM = (uint32_t)(BM * NCTA) >> 4;
             uint32_t idesc;
-            if (C::MX) idesc = (1u << 23) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
-            else idesc = (1u << 4) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
-            for (int pos = blockIdx.x; pos < positions && ok; pos += gridDim.x) {
+            if (C::MX) idesc = (1u << 23) | ((uint32_t)(BN >> 3) << 17) | (MDIM << 24);
+            else idesc = (1u << 4) | ((uint32_t)(BN >> 3) << 17) | (MDIM << 24);
+            for (int pos = unit; pos < positions && ok; pos += units) {
                 for (int t = 0; t < p.terms && ok; ++t) {
                     if (C::MX) {
+                        const long long tw = TCLK();
                         if (!mbar_wait(bar_tempty(0), bphase ^ 1u, ctl, 201)) { ok = false; break; }
+                        TADD(1, tw);
                         tc_fence_after();
                     }
                     for (int ks = 0; ks < kstages; ++ks) {
+                        const long long tw2 = TCLK();
                         if (!mbar_wait(bar_full(stage), phase, ctl, 202)) { ok = false; break; }
+                        TADD(2, tw2);
                         tc_fence_after();
                         const uint64_t adesc = make_kmajor_sw128_desc(base + C::OFF_A + stage * C::A_BYTES);
                         const uint64_t bdesc = make_kmajor_sw128_desc(base + C::OFF_B + stage * C::B_BYTES);
@@ -300,95 +261,131 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                             const uint32_t sf = base + C::OFF_SF + stage * C::SF_STAGE_BYTES;
                             const uint32_t tsfa = tmem_base + BN + stage * C::SF_COLS;
                             const uint32_t tsfb = tsfa + 4;
-                            tc_cp_32x128b_warpx4(tsfa, make_sf_desc(sf));
+#ifndef FMM_EXP_NO_CP
+                            tc_cp_32x128b_warpx4<NCTA>(tsfa, make_sf_desc(sf));
 #pragma unroll
-                            for (int h = 0; h < BN / 128; ++h) tc_cp_32x128b_warpx4(tsfb + 4 * h, make_sf_desc(sf + 512 + h * 512));
+                            for (int h = 0; h < C::SFB_ATOMS; ++h)
+                                tc_cp_32x128b_warpx4<NCTA>(tsfb + 4 * h, make_sf_desc(sf + 512 + h * 512));
+#endif
 #pragma unroll
                             for (int j = 0; j < BK / 32; ++j) {
                                 const uint32_t id = idesc | ((uint32_t)j << 29) | ((uint32_t)j << 4);
-                                mma_mxf8(tmem_base, adesc + 2 * j, bdesc + 2 * j, id, (ks > 0 || j > 0) ? 1u : 0u, tsfa, tsfb);
+                                mma_mxf8<NCTA>(tmem_base, adesc + 2 * j, bdesc + 2 * j, id, (ks > 0 || j > 0) ? 1u : 0u, tsfa, tsfb);
                             }
                         } else {
 #pragma unroll
                             for (int g = 0; g < C::KB_PER_STAGE; ++g) {
+                                const long long tw3 = TCLK();
                                 if (!mbar_wait(bar_tempty(buf), bphase ^ 1u, ctl, 203)) { ok = false; break; }
+                                TADD(1, tw3);
                                 tc_fence_after();
 #pragma unroll
                                 for (int j = 0; j < BLK / 32; ++j) {
                                     const int jj = g * (BLK / 32) + j;
-                                    mma_f8f6f4(tmem_base + buf * BN, adesc + 2 * jj, bdesc + 2 * jj, idesc, j > 0 ? 1u : 0u);
+                                    mma_f8f6f4<NCTA>(tmem_base + buf * BN, adesc + 2 * jj, bdesc + 2 * jj, idesc, j > 0 ? 1u : 0u);
                                 }
-                                tc_commit(bar_tfull(buf));
+                                tc_commit<NCTA>(bar_tfull(buf));
                                 if (++buf == C::ACC_BUFS) { buf = 0; bphase ^= 1u; }
                             }
                             if (!ok) break;
                         }
-                        tc_commit(bar_empty(stage));
+                        tc_commit<NCTA>(bar_empty(stage));
                         if (++stage == C::STAGES) { stage = 0; phase ^= 1u; }
                     }
-                    if (C::MX && ok) { tc_commit(bar_tfull(0)); bphase ^= 1u; }
+                    if (C::MX && ok) { tc_commit<NCTA>(bar_tfull(0)); bphase ^= 1u; }
                 }
             }
         }
+    }
     } else {
         // ------------------------------------------------------------------ epilogue warps
-        const int e = warp - 2;
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(REGS_EPI));
+        const int e = warp - EPI_WARP0;
         const int q = warp & 3;            // TMEM lane quadrant this warp may access
         const int h = e >> 2;              // column half
         const uint32_t stg = base + C::OFF_STG + e * STAGING_BUFS * STAGING_BYTES;
         uint8_t* stg_ptr = base_ptr + C::OFF_STG + e * STAGING_BUFS * STAGING_BYTES;
         const uint32_t lane_taddr = tmem_base + ((uint32_t)(q * 32) << 16) + h * C::CW;
+        // the accumulator-free signal goes to the MMA issuer, which lives in the even CTA
+        auto release_acc = [&](int b) {
+            if (NCTA == 2) mbar_arrive_cluster(bar_tempty(b) & PEER_BIT_MASK); else mbar_arrive(bar_tempty(b));
+        };
         int buf = 0; uint32_t bphase = 0;
         int ss = 0; uint32_t sphase = 0;
         uint32_t store_cnt = 0;
         bool ok = true;
-        float acc[C::CW];
-        for (int pos = blockIdx.x; pos < positions && ok; pos += gridDim.x) {
+        uint32_t accu[C::MX ? C::CW : 1];               // UE8M0: raw fp32 bits drained from TMEM
+        unsigned long long acc2[C::MX ? 1 : C::CW / 2]; // FP32: promoted accumulators, two columns per register pair
+        for (int pos = unit; pos < positions && ok; pos += units) {
             const int tm = pos / tiles_n, tn = pos % tiles_n;
+            const int row_in_leaf = (tm * NCTA + cta_rank) * BM + q * 32;
             for (int t = 0; t < p.terms && ok; ++t) {
                 if (C::MX) {
+                    const long long tw = TCLK();
                     if (!mbar_wait_warp(bar_tfull(0), bphase, ctl, 301)) { ok = false; break; }
+                    TADD(3, tw);
                     tc_fence_after();
 #pragma unroll
-                    for (int c = 0; c < C::CW / 32; ++c) tmem_ld32(lane_taddr + c * 32, &acc[c * 32]);
+                    for (int c = 0; c < C::CW / 32; ++c) tmem_ld32(lane_taddr + c * 32, &accu[c * 32]);
                     tmem_ld_wait();
                     tc_fence_before();
                     __syncwarp();
-                    if (lane == 0) mbar_arrive(bar_tempty(0));
+                    if (lane == 0) release_acc(0);
                     bphase ^= 1u;
                 } else {
 #pragma unroll
-                    for (int i = 0; i < C::CW; ++i) acc[i] = 0.0f;
+                    for (int i = 0; i < C::CW / 2; ++i) acc2[i] = 0ull;
                     const float* sa_row = reinterpret_cast<const float*>(p.sa + (long long)t * p.sa_term) +
-                                          (long long)(tm * BM + q * 32 + lane) * nkb;
+                                          (long long)(row_in_leaf + lane) * nkb;
+                    // row scales are prefetched PF stages ahead (each thread walks its own row of the scale matrix)
+                    constexpr int PF = (C::KB_PER_STAGE >= 4) ? 1 : 2;
+                    float sa_q[PF + 1][C::KB_PER_STAGE];
+#pragma unroll
+                    for (int d = 0; d < PF; ++d)
+#pragma unroll
+                        for (int g = 0; g < C::KB_PER_STAGE; ++g)
+                            sa_q[d][g] = (d < kstages) ? __ldg(sa_row + d * C::KB_PER_STAGE + g) : 0.0f;
                     for (int ks = 0; ks < kstages && ok; ++ks) {
+#pragma unroll
+                        for (int g = 0; g < C::KB_PER_STAGE; ++g)
+                            sa_q[PF][g] = (ks + PF < kstages) ? __ldg(sa_row + (ks + PF) * C::KB_PER_STAGE + g) : 0.0f;
                         if (!mbar_wait_warp(bar_sfull(ss), sphase, ctl, 302)) { ok = false; break; }
                         float sa[C::KB_PER_STAGE];
 #pragma unroll
-                        for (int g = 0; g < C::KB_PER_STAGE; ++g) sa[g] = __ldg(sa_row + ks * C::KB_PER_STAGE + g);
-                        const float* sbs = reinterpret_cast<const float*>(base_ptr + C::OFF_SB + ss * C::SB_STAGE_BYTES);
+                        for (int g = 0; g < C::KB_PER_STAGE; ++g) {
+                            sa[g] = sa_q[0][g];
+#pragma unroll
+                            for (int d = 0; d < PF; ++d) sa_q[d][g] = sa_q[d + 1][g];
+                        }
+                        const uint8_t* sbs = base_ptr + C::OFF_SB + ss * C::SB_STAGE_BYTES;
 #pragma unroll
                         for (int g = 0; g < C::KB_PER_STAGE; ++g) {
+                            const long long tw = TCLK();
                             if (!mbar_wait_warp(bar_tfull(buf), bphase, ctl, 303)) { ok = false; break; }
+                            TADD(3, tw);
                             tc_fence_after();
-                            const float* sbg = sbs + g * BN + h * C::CW;
+                            const ulonglong2* sbg = reinterpret_cast<const ulonglong2*>(sbs + (g * BN + h * C::CW) * 4);
+                            const unsigned long long sa2 = pack2(sa[g], sa[g]);
+                            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + buf * BN + h * C::CW;
+                            uint32_t tmp[32];
 #pragma unroll
                             for (int c = 0; c < C::CW / 32; ++c) {
-                                float tmp[32];
-                                tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + buf * BN + h * C::CW + c * 32, tmp);
+                                tmem_ld32(taddr + c * 32, tmp);      // a TMEM load round trip is a few tens of cycles
                                 tmem_ld_wait();
+                                if (c + 1 == C::CW / 32) {
+                                    // the last chunk is in registers: hand the TMEM buffer back before the arithmetic
+                                    tc_fence_before();
+                                    __syncwarp();
+                                    if (lane == 0) release_acc(buf);
+                                }
 #pragma unroll
-                                for (int i = 0; i < 32; i += 4) {
-                                    const float4 s4 = *reinterpret_cast<const float4*>(sbg + c * 32 + i);
-                                    acc[c * 32 + i + 0] = fmaf(tmp[i + 0], sa[g] * s4.x, acc[c * 32 + i + 0]);
-                                    acc[c * 32 + i + 1] = fmaf(tmp[i + 1], sa[g] * s4.y, acc[c * 32 + i + 1]);
-                                    acc[c * 32 + i + 2] = fmaf(tmp[i + 2], sa[g] * s4.z, acc[c * 32 + i + 2]);
-                                    acc[c * 32 + i + 3] = fmaf(tmp[i + 3], sa[g] * s4.w, acc[c * 32 + i + 3]);
+                                for (int i = 0; i < 8; ++i) {
+                                    const ulonglong2 s4 = sbg[c * 8 + i];        // four column scales
+                                    const uint32_t* tp = tmp + 4 * i;
+                                    acc2[c * 16 + 2 * i] = fma2(pack2u(tp[0], tp[1]), mul2(sa2, s4.x), acc2[c * 16 + 2 * i]);
+                                    acc2[c * 16 + 2 * i + 1] = fma2(pack2u(tp[2], tp[3]), mul2(sa2, s4.y), acc2[c * 16 + 2 * i + 1]);
                                 }
                             }
-                            tc_fence_before();
-                            __syncwarp();
-                            if (lane == 0) mbar_arrive(bar_tempty(buf));
                             if (++buf == C::ACC_BUFS) { buf = 0; bphase ^= 1u; }
                         }
                         __syncwarp();
@@ -398,24 +395,31 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                     if (!ok) break;
                 }
                 // ---- post-addition: W-weighted scatter of this product into its C blocks
+                const long long t_out = TCLK();
                 const int o0 = p.out_start[t], o1 = p.out_start[t + 1];
                 if (lane == 0) bulk_wait<0>();     // the previous term's writes to these tiles have landed
                 __syncwarp();
                 for (int o = o0; o < o1; ++o) {
                     const FmmOutEntry ent = p.out[o];
-                    const int row0 = ent.row_off * p.m + tm * BM + q * 32;
+                    const int row0 = ent.row_off * p.m + row_in_leaf;
                     const int col0 = ent.col_off * p.n + tn * BN + h * C::CW;
 #pragma unroll
                     for (int c = 0; c < C::CW / 32; ++c) {
                         const uint32_t b = store_cnt & (STAGING_BUFS - 1);
-                        if (lane == 0) bulk_wait_read<STAGING_BUFS - 1>();
+                        if (lane == 0) bulk_wait_read<STAGING_BUFS - 1>();   // the buffer about to be rewritten has been read
                         __syncwarp();
                         uint8_t* dst = stg_ptr + b * STAGING_BYTES + lane * 128;
 #pragma unroll
                         for (int i4 = 0; i4 < 8; ++i4) {
                             float4 v;
-                            v.x = acc[c * 32 + i4 * 4 + 0] * ent.w; v.y = acc[c * 32 + i4 * 4 + 1] * ent.w;
-                            v.z = acc[c * 32 + i4 * 4 + 2] * ent.w; v.w = acc[c * 32 + i4 * 4 + 3] * ent.w;
+                            if (C::MX) {
+                                v.x = __uint_as_float(accu[c * 32 + i4 * 4 + 0]); v.y = __uint_as_float(accu[c * 32 + i4 * 4 + 1]);
+                                v.z = __uint_as_float(accu[c * 32 + i4 * 4 + 2]); v.w = __uint_as_float(accu[c * 32 + i4 * 4 + 3]);
+                            } else {
+                                unpack2(acc2[c * 16 + i4 * 2], v.x, v.y);
+                                unpack2(acc2[c * 16 + i4 * 2 + 1], v.z, v.w);
+                            }
+                            v.x *= ent.w; v.y *= ent.w; v.z *= ent.w; v.w *= ent.w;
                             *reinterpret_cast<float4*>(dst + ((i4 ^ (lane & 7)) << 4)) = v;
                         }
                         fence_proxy_async();
@@ -428,11 +432,19 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                         ++store_cnt;
                     }
                 }
+                TADD(4, t_out);
             }
         }
         if (lane == 0) bulk_wait<0>();
     }
 
+#ifdef FMM_TIMING
+    if (blockIdx.x == 0 && lane == 0 && (warp <= 1 || warp == EPI_WARP0)) {
+        long long* dst = reinterpret_cast<long long*>(p.status + 8) + (warp <= 1 ? warp : 2) * 8;
+        for (int i = 0; i < 7; ++i) dst[i] = tim[i];
+        dst[7] = clock64() - t_kernel;
+    }
+#endif
     // ---------------------------------------------------------------------- teardown
     if (*abort_flag) {
         // let copies that are still in flight towards this CTA's shared memory land
@@ -441,10 +453,11 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     }
     tc_fence_before();
     __syncthreads();
+    if (NCTA == 2) cluster_sync();      // the peer no longer reads this CTA's shared memory or signals its barriers
     if (warp == 1) {
         __syncwarp();
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512) : "memory");
+        tmem_dealloc<NCTA>(tmem_base, 512);
     }
 }
 
@@ -468,7 +481,7 @@ EncodeTiledFn get_encode_fn()
 }
 
 bool make_map_2d(CUtensorMap* tm, CUtensorMapDataType dt, int elt_bytes, const void* ptr, uint64_t inner, uint64_t outer,
-                 uint32_t box_inner, uint32_t box_outer)
+                 uint32_t box_inner, uint32_t box_outer, CUtensorMapSwizzle swz)
 {
     EncodeTiledFn fn = get_encode_fn();
     if (!fn) return false;
@@ -477,20 +490,29 @@ bool make_map_2d(CUtensorMap* tm, CUtensorMapDataType dt, int elt_bytes, const v
     cuuint32_t box[2] = {box_inner, box_outer};
     cuuint32_t estr[2] = {1, 1};
     return fn(tm, dt, 2, const_cast<void*>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+              swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int BN, int MODE, int BLK>
+template <int BN, int MODE, int BLK, int NCTA>
 fmm_status_t launch(const GemmParams& g, cudaStream_t st)
 {
-    using C = Cfg<BN, MODE, BLK>;
-    CUtensorMap tmA, tmB, tmC;
-    if (!make_map_2d(&tmA, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, g.qa, (uint64_t)g.k, (uint64_t)g.terms * g.m, BK, BM)) return FMM_ERR_CUDA;
-    if (!make_map_2d(&tmB, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, g.qb, (uint64_t)g.k, (uint64_t)g.terms * g.n, BK, BN)) return FMM_ERR_CUDA;
-    if (!make_map_2d(&tmC, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, g.C, (uint64_t)g.Nfull, (uint64_t)g.Mfull, 32, 32)) return FMM_ERR_CUDA;
+    using C = Cfg<BN, MODE, BLK, NCTA>;
+    CUtensorMap tmA, tmB, tmC, tmSFA, tmSFB;
+    const CUtensorMapSwizzle SW = CU_TENSOR_MAP_SWIZZLE_128B;
+    if (!make_map_2d(&tmA, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, g.qa, (uint64_t)g.k, (uint64_t)g.terms * g.m, BK, BM, SW)) return FMM_ERR_CUDA;
+    if (!make_map_2d(&tmB, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, g.qb, (uint64_t)g.k, (uint64_t)g.terms * g.n, BK, C::BROWS, SW)) return FMM_ERR_CUDA;
+    if (!make_map_2d(&tmC, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, g.C, (uint64_t)g.Nfull, (uint64_t)g.Mfull, 32, 32, SW)) return FMM_ERR_CUDA;
+    if (C::MX) {
+        // scale tiles as rows of 128 uint32 (one 512-byte atom per row)
+        const uint64_t atoms_a = (uint64_t)g.terms * (g.k / 128) * (g.m / 128), atoms_b = (uint64_t)g.terms * (g.k / 128) * (g.n / 128);
+        if (!make_map_2d(&tmSFA, CU_TENSOR_MAP_DATA_TYPE_UINT32, 4, g.sa, 128, atoms_a, 128, 1, CU_TENSOR_MAP_SWIZZLE_NONE)) return FMM_ERR_CUDA;
+        if (!make_map_2d(&tmSFB, CU_TENSOR_MAP_DATA_TYPE_UINT32, 4, g.sb, 128, atoms_b, 128, C::SFB_ATOMS, CU_TENSOR_MAP_SWIZZLE_NONE)) return FMM_ERR_CUDA;
+    } else {
+        tmSFA = tmA; tmSFB = tmB;       // unused in this mode
+    }
     static bool attr_set = false;
     if (!attr_set) {
-        if (cudaFuncSetAttribute(fmm_gemm_kernel<BN, MODE, BLK>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES) != cudaSuccess) {
+        if (cudaFuncSetAttribute(fmm_gemm_kernel<BN, MODE, BLK, NCTA>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES) != cudaSuccess) {
             cudaGetLastError();
             return FMM_ERR_CUDA;
         }
@@ -499,30 +521,47 @@ fmm_status_t launch(const GemmParams& g, cudaStream_t st)
     int dev = 0, sms = 0;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    const int positions = (g.m / BM) * (g.n / BN);
-    const int grid = positions < sms ? positions : sms;
+    const int positions = (g.m / (BM * NCTA)) * (g.n / BN);
+    const int max_units = sms / NCTA;
+    const int units = positions < max_units ? positions : max_units;
     KParams kp;
     kp.sa = static_cast<const uint8_t*>(g.sa); kp.sb = static_cast<const uint8_t*>(g.sb);
     kp.sa_term = g.sa_term; kp.sb_term = g.sb_term;
     kp.m = g.m; kp.n = g.n; kp.k = g.k; kp.terms = g.terms;
     kp.out_start = g.out_start; kp.out = g.out; kp.status = g.status;
-    fmm_gemm_kernel<BN, MODE, BLK><<<grid, NUM_THREADS, C::SMEM_BYTES, st>>>(tmA, tmB, tmC, kp);
-    return cudaGetLastError() == cudaSuccess ? FMM_OK : FMM_ERR_CUDA;
+
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3((unsigned)(units * NCTA), 1, 1);
+    cfg.blockDim = dim3(NUM_THREADS, 1, 1);
+    cfg.dynamicSmemBytes = C::SMEM_BYTES;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = NCTA; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    cudaError_t ce = cudaLaunchKernelEx(&cfg, fmm_gemm_kernel<BN, MODE, BLK, NCTA>, tmA, tmB, tmC, tmSFA, tmSFB, kp);
+    if (ce != cudaSuccess) { cudaGetLastError(); return FMM_ERR_CUDA; }
+    return FMM_OK;
+}
+
+template <int MODE, int BLK>
+fmm_status_t launch_shape(const GemmParams& g, cudaStream_t st)
+{
+    // pairs of CTAs with 256 x 256 tiles whenever the leaf shape allows it; single CTAs otherwise
+    if ((g.m % 256) == 0 && (g.n % 256) == 0) return launch<256, MODE, BLK, 2>(g, st);
+    if ((g.n % 256) == 0) return launch<256, MODE, BLK, 1>(g, st);
+    return launch<128, MODE, BLK, 1>(g, st);
 }
 
 }  // namespace
 
 fmm_status_t fmm_launch_gemm(const GemmParams& g, int blk, int mode, cudaStream_t st, int* launches)
 {
-    const bool wide = (g.n % 256) == 0;
     fmm_status_t s;
-    if (mode == FMM_SCALE_UE8M0_CEIL) {
-        s = wide ? launch<256, FMM_SCALE_UE8M0_CEIL, 32>(g, st) : launch<128, FMM_SCALE_UE8M0_CEIL, 32>(g, st);
-    } else if (blk == 32) {
-        s = wide ? launch<256, FMM_SCALE_FP32_AMAX_DIV_448, 32>(g, st) : launch<128, FMM_SCALE_FP32_AMAX_DIV_448, 32>(g, st);
-    } else {
-        s = wide ? launch<256, FMM_SCALE_FP32_AMAX_DIV_448, 128>(g, st) : launch<128, FMM_SCALE_FP32_AMAX_DIV_448, 128>(g, st);
-    }
+    if (mode == FMM_SCALE_UE8M0_CEIL) s = launch_shape<FMM_SCALE_UE8M0_CEIL, 32>(g, st);
+    else if (blk == 32) s = launch_shape<FMM_SCALE_FP32_AMAX_DIV_448, 32>(g, st);
+    else s = launch_shape<FMM_SCALE_FP32_AMAX_DIV_448, 128>(g, st);
     if (s == FMM_OK && launches) *launches += 1;
     return s;
 }

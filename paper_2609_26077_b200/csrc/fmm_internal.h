@@ -34,7 +34,7 @@ struct fmm_plan {
     int terms;
     int device;
     // device tables
-    int* d_status;            // [4] status words
+    int* d_status;            // [64] status words (word 0: first bounded wait that gave up)
     int* d_out_start;         // [terms + 1]
     FmmOutEntry* d_out;       // [total entries], block offsets in units of leaf blocks (scaled at launch)
     int n_out_total;

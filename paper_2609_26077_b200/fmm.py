@@ -8,7 +8,7 @@ import os
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libfmm_b200.so")
+LIB_PATH = os.environ.get("FMM_B200_LIB", os.path.join(_HERE, "libfmm_b200.so"))   # override: experiment builds
 
 FMM_OK = 0
 STATUS_NAMES = ["FMM_OK", "FMM_ERR_INVALID_ARG", "FMM_ERR_SHAPE", "FMM_ERR_NOT_EXACT", "FMM_ERR_WORKSPACE",
@@ -186,8 +186,8 @@ class Plan:
                 codes = codes.T
         else:
             rows, nkb = sr, sc
-            tiles = host[so:so + rows * nkb].reshape(rows // 128, nkb // 4, 32, 4, 4)   # [tile_r, tile_k, r%32, (r%128)/32, kb%4]
-            scales = tiles.transpose(0, 3, 2, 1, 4).reshape(rows, nkb)
+            tiles = host[so:so + rows * nkb].reshape(nkb // 4, rows // 128, 32, 4, 4)   # [kb/4, r/128, r%32, (r%128)/32, kb%4]
+            scales = tiles.transpose(1, 3, 2, 0, 4).reshape(rows, nkb)
             if side == "B":
                 codes = codes.T
                 scales = scales.T
