@@ -135,6 +135,24 @@ fmm_status_t fmm_error_stats(const float* C, const double* Cref, int64_t M, int6
                              double* out3, void* scratch, size_t scratch_bytes, void* cuda_stream);
 size_t fmm_error_stats_scratch_bytes(void);
 
+/* (No counterpart in the paper: a convenience for restricted callers.)
+ * Same result as fmm_error_stats, for callers that are not allowed to allocate device memory at all -
+ * code running inside a service whose memory pool is fixed up front, a plugin that must not touch the
+ * host application's allocator, or a routine invoked where cudaMalloc would synchronise the device at a
+ * bad moment.  The block partials go to a fixed 24 KB array compiled into the library (1024 slots of
+ * three doubles, resident on every GPU that loads the library), so the call takes no scratch argument
+ * and performs no allocation of any kind; C, Cref and out3 are still the caller's.
+ *   Limit: M * N <= fmm_error_stats_noalloc_max_elements() (2^28, e.g. 16384 x 16384) and M * N even;
+ *   larger problems are refused with FMM_ERR_SHAPE - use fmm_error_stats with your own scratch.
+ *   The first call on each device looks up the array's device address (with that device current) and
+ *   remembers it; make that first call outside any stream capture.
+ *   All calls on a device share the one array.  Every slot is rewritten by each call, so stale contents
+ *   are harmless, but two calls whose kernels overlap on the GPU (different streams, no ordering
+ *   between them) would overwrite each other's partials: order such calls. */
+fmm_status_t fmm_error_stats_noalloc(const float* C, const double* Cref, int64_t M, int64_t N,
+                                     double* out3, void* cuda_stream);
+int64_t fmm_error_stats_noalloc_max_elements(void);
+
 /* Reads the plan's device status word (synchronises the device).  *code == 0: no bounded wait has
  * given up since plan creation; otherwise a kernel-specific location code, and the results of the
  * call that set it are invalid.  Returns FMM_ERR_DEVICE_TIMEOUT when *code != 0. */

@@ -4,11 +4,18 @@
 //   fmm_error_stats   : sum (C - Cref)^2, sum Cref^2, max |C - Cref| with fp64 accumulation,
 //                       warp-shuffle + shared-memory tree per block, fixed block partition and a
 //                       single-block second stage, hence bit-reproducible.
+#include <mutex>
 #include "fmm_internal.h"
+
+// Scratch of fmm_error_stats_noalloc: one partial triple per reduction block.  It lives in the
+// library image, so every GPU that loads the library carries these 24 KB until the process exits.
+// In host code this name is only a stand-in for the symbol; the device address comes from
+// cudaGetSymbolAddress (see noalloc_scratch below).
+static __device__ __align__(256) double g_noalloc_partials[3 * 1024];
 
 namespace {
 
-constexpr int STAT_BLOCKS = 1024;
+constexpr int STAT_BLOCKS = 1024;     // also the number of slots of g_noalloc_partials
 constexpr int STAT_THREADS = 256;
 
 __device__ __forceinline__ void warp_reduce3(double& a, double& b, double& c)
@@ -150,5 +157,52 @@ fmm_status_t fmm_ref_gemm_fp64(const float* A, const float* B, double* Cref, int
     ref_gemm_fp64_kernel<<<grid, 256, 0, reinterpret_cast<cudaStream_t>(stream)>>>(A, B, Cref, M, N, K);
     return cudaGetLastError() == cudaSuccess ? FMM_OK : FMM_ERR_CUDA;
 }
+
+// ---- variant of fmm_error_stats for callers that cannot allocate device memory ----------------
+namespace {
+constexpr int NOALLOC_MAX_DEVICES = 64;
+constexpr int64_t NOALLOC_MAX_ELEMS = (int64_t)1 << 28;    // 1024 scratch slots x at most 2^18 elements each
+std::mutex g_noalloc_mutex;
+double* g_noalloc_ptr[NOALLOC_MAX_DEVICES] = {nullptr};
+
+// Device address of the static scratch on the current device, resolved once per device.
+fmm_status_t noalloc_scratch(double** out)
+{
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return FMM_ERR_CUDA; }
+    if (dev < 0 || dev >= NOALLOC_MAX_DEVICES) return FMM_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+    if (!g_noalloc_ptr[dev]) {
+        double* ptr = nullptr;
+        if (cudaGetSymbolAddress((void**)&ptr, g_noalloc_partials) != cudaSuccess || !ptr) {
+            cudaGetLastError();
+            return FMM_ERR_CUDA;
+        }
+        g_noalloc_ptr[dev] = ptr;
+    }
+    *out = g_noalloc_ptr[dev];
+    return FMM_OK;
+}
+}  // namespace
+
+fmm_status_t fmm_error_stats_noalloc(const float* C, const double* Cref, int64_t M, int64_t N, double* out3,
+                                     void* stream)
+{
+    if (!C || !Cref || !out3) return FMM_ERR_INVALID_ARG;
+    if (M <= 0 || N <= 0 || ((M * N) & 1)) return FMM_ERR_SHAPE;
+    if (M > NOALLOC_MAX_ELEMS || N > NOALLOC_MAX_ELEMS || M * N > NOALLOC_MAX_ELEMS) return FMM_ERR_SHAPE;
+    if (((uintptr_t)C & 7) || ((uintptr_t)Cref & 15)) return FMM_ERR_INVALID_ARG;
+    double* partial = nullptr;
+    fmm_status_t s = noalloc_scratch(&partial);
+    if (s != FMM_OK) return s;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    // every one of the STAT_BLOCKS slots is rewritten by the first kernel, so nothing left behind by
+    // an earlier call is ever read and no clearing is needed
+    error_partial_kernel<<<STAT_BLOCKS, STAT_THREADS, 0, st>>>(C, Cref, M * N, partial);
+    error_final_kernel<<<1, STAT_THREADS, 0, st>>>(partial, STAT_BLOCKS, out3);
+    return cudaGetLastError() == cudaSuccess ? FMM_OK : FMM_ERR_CUDA;
+}
+
+int64_t fmm_error_stats_noalloc_max_elements(void) { return NOALLOC_MAX_ELEMS; }
 
 }  // extern "C"

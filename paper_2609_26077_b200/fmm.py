@@ -18,7 +18,8 @@ SCALE_MODES = {"fp32": SCALE_FP32, "ue8m0": SCALE_UE8M0}
 
 EXPORTS = ["fmm_plan_create", "fmm_plan_destroy", "fmm_workspace_bytes", "fmm_matmul", "fmm_encode_only",
            "fmm_multiply_only", "fmm_quantized_view", "fmm_ref_gemm_fp64", "fmm_error_stats",
-           "fmm_error_stats_scratch_bytes", "fmm_device_status", "fmm_phi_gamma", "fmm_brent_residual",
+           "fmm_error_stats_scratch_bytes", "fmm_error_stats_noalloc", "fmm_error_stats_noalloc_max_elements",
+           "fmm_device_status", "fmm_phi_gamma", "fmm_brent_residual",
            "fmm_last_launch_count", "fmm_status_string"]
 
 
@@ -47,6 +48,7 @@ def lib():
         L.fmm_status_string.restype = C.c_char_p
         L.fmm_status_string.argtypes = [C.c_int]
         L.fmm_error_stats_scratch_bytes.restype = C.c_size_t
+        L.fmm_error_stats_noalloc_max_elements.restype = C.c_int64
         for name in EXPORTS:
             getattr(L, name)
         _lib = L
@@ -230,6 +232,15 @@ def fmm_error_stats(Cm, Cref, out3=None, stream=None):
     sc = _scratch[key]
     _check(lib().fmm_error_stats(_dev_ptr(Cm), _dev_ptr(Cref), C.c_int64(M), C.c_int64(N), _dev_ptr(out3),
                                  _dev_ptr(sc), C.c_size_t(sc.numel()), _stream_ptr(stream)), "fmm_error_stats")
+    return out3
+
+
+def fmm_error_stats_noalloc(Cm, Cref, out3, stream=None):
+    """fmm_error_stats_noalloc: same statistics, block partials in the library's built-in scratch.
+    Nothing is allocated here either: the caller supplies out3 (3 doubles on the device)."""
+    M, N = Cm.shape
+    _check(lib().fmm_error_stats_noalloc(_dev_ptr(Cm), _dev_ptr(Cref), C.c_int64(M), C.c_int64(N), _dev_ptr(out3),
+                                         _stream_ptr(stream)), "fmm_error_stats_noalloc")
     return out3
 
 
