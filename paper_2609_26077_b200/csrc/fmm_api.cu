@@ -103,9 +103,33 @@ fmm_status_t encode_side(fmm_plan* plan, const FmmLayout& L, char* ws, const flo
     e.amax_floor = plan->qp.amax_floor;
     fmm_status_t s;
     if (lv == 0) {
+        // Plain quantization of the matrix itself.  The matrix is cut into four panels (row panels of A,
+        // column panels of B) that are handled like four "combinations" with identity coefficients, so
+        // each thread keeps four independent loads in flight; the outputs land where the unsplit
+        // matrix would put them.
+        const bool panels = b_side ? (cols % 256 == 0) : (rows % 4 == 0);
         e.in = X; e.in_batch_stride = 0; e.ld = cols; e.batch = 1;
-        e.rows = (int)rows; e.cols = (int)cols; e.nq = 1; e.R = 1;
-        e.coef[0][0] = 1.0f;
+        if (panels) {
+            e.nq = 4; e.R = 4;
+            for (int r = 0; r < 4; ++r) e.coef[r][r] = 1.0f;
+            if (b_side) {
+                e.rows = (int)rows; e.cols = (int)(cols / 4);
+                for (int j = 0; j < 4; ++j) e.qoff[j] = (int64_t)j * (cols / 4);
+                e.s_step = (int)(cols / 4); e.s_ld = (int)cols; e.sf_blocks = (int)(cols / 128);
+            } else {
+                e.rows = (int)(rows / 4); e.cols = (int)cols;
+                for (int j = 0; j < 4; ++j) e.qoff[j] = (int64_t)j * (rows / 4) * cols;
+                e.s_step = (int)(rows / 4); e.s_ld = 0; e.sf_blocks = (int)(rows / 128);
+            }
+            // fp32 scales of the A side and all codes are contiguous per panel; shared arrays otherwise
+            const bool fp32 = mode == FMM_SCALE_FP32_AMAX_DIV_448;
+            if (!b_side && fp32) { e.s_term_stride = (int64_t)(rows / 4) * (cols / blk) * 4; e.s_step = 0; }
+            else e.s_term_stride = 0;
+        } else {
+            e.rows = (int)rows; e.cols = (int)cols; e.nq = 1; e.R = 1;
+            e.coef[0][0] = 1.0f;
+            e.s_step = 0; e.s_ld = (int)cols; e.sf_blocks = (int)((b_side ? cols : rows) / 128);
+        }
     } else {
         const float* cur = X;
         int64_t cur_rows = rows, cur_cols = cols, cur_ld = cols, cur_stride = 0;
@@ -125,7 +149,9 @@ fmm_status_t encode_side(fmm_plan* plan, const FmmLayout& L, char* ws, const flo
         }
         e.in = cur; e.in_batch_stride = cur_stride; e.ld = cur_ld; e.batch = batch;
         e.rows = (int)(cur_rows / 2); e.cols = (int)(cur_cols / 2); e.nq = 4; e.R = R;
+        e.qoff[0] = 0; e.qoff[1] = e.cols; e.qoff[2] = (int64_t)e.rows * e.ld; e.qoff[3] = (int64_t)e.rows * e.ld + e.cols;
         fill_coef(e.coef, coef, R);
+        e.s_step = 0; e.s_ld = e.cols; e.sf_blocks = (b_side ? e.cols : e.rows) / 128;
     }
     s = b_side ? fmm_launch_encode_b(e, blk, mode, st) : fmm_launch_encode_a(e, blk, mode, st);
     if (s == FMM_OK) plan->last_launches++;

@@ -77,7 +77,6 @@ __global__ void __launch_bounds__(256) encode_a_kernel(const EncodeParams p)
     const int chunks = p.cols / 128;
     const int nkb = p.cols / BLK;
     const int64_t units = (int64_t)p.batch * p.rows * chunks;
-    const int64_t qoff[4] = {0, (int64_t)p.cols, (int64_t)p.rows * p.ld, (int64_t)p.rows * p.ld + p.cols};
     const int64_t term_codes = (int64_t)p.rows * p.cols;
     const bool b2 = lane & 4, b1 = lane & 2, b0 = lane & 1;
     const int my_r = lane & 7;
@@ -92,7 +91,7 @@ __global__ void __launch_bounds__(256) encode_a_kernel(const EncodeParams p)
 #pragma unroll
         for (int j = 0; j < 4; ++j)
             if (j < p.nq) {
-                const float4 x = __ldcs(reinterpret_cast<const float4*>(base + qoff[j]));
+                const float4 x = __ldcs(reinterpret_cast<const float4*>(base + p.qoff[j]));
                 xl[j] = pack2(x.x, x.y); xh[j] = pack2(x.z, x.w);
             }
 
@@ -165,8 +164,9 @@ __global__ void __launch_bounds__(256) encode_a_kernel(const EncodeParams p)
             wv |= __shfl_xor_sync(FULL, wv, 16);
             if (lane < 8 && lane < p.R) {
                 char* so = reinterpret_cast<char*>(p.s_out) + ((int64_t)b * p.R + lane) * p.s_term_stride;
-                const int64_t tile = (int64_t)c * (p.rows >> 7) + (i >> 7);
-                *reinterpret_cast<uint32_t*>(so + tile * 512 + (i & 31) * 16 + ((i & 127) >> 5) * 4) = wv;
+                const int ig = i + lane * p.s_step;            // row inside the scale-tile array
+                const int64_t tile = (int64_t)c * p.sf_blocks + (ig >> 7);
+                *reinterpret_cast<uint32_t*>(so + tile * 512 + (ig & 31) * 16 + ((ig & 127) >> 5) * 4) = wv;
             }
         }
     }
@@ -180,15 +180,16 @@ __global__ void __launch_bounds__(256) encode_a_kernel(const EncodeParams p)
 // lanes of a block fill one 32-byte sector.  BLK == 128 takes a second pass over the four
 // 32-element sub-blocks (served by L1/L2).
 template <int MODE>
-__device__ __forceinline__ void store_b_scale(const EncodeParams& p, int64_t t, int j, int kb, int kc,
+__device__ __forceinline__ void store_b_scale(const EncodeParams& p, int64_t t, int r, int j, int kb, int kc,
                                               float s, uint32_t e8word, bool last_of_word)
 {
     char* so = reinterpret_cast<char*>(p.s_out) + t * p.s_term_stride;
+    const int jg = j + r * p.s_step;                   // column inside the scale array
     if (MODE == FMM_SCALE_FP32_AMAX_DIV_448) {
-        reinterpret_cast<float*>(so)[(int64_t)kb * p.cols + j] = s;
+        reinterpret_cast<float*>(so)[(int64_t)kb * p.s_ld + jg] = s;
     } else if (last_of_word) {
-        const int64_t tile = (int64_t)kc * (p.cols >> 7) + (j >> 7);
-        *reinterpret_cast<uint32_t*>(so + tile * 512 + (j & 31) * 16 + ((j & 127) >> 5) * 4) = e8word;
+        const int64_t tile = (int64_t)kc * p.sf_blocks + (jg >> 7);
+        *reinterpret_cast<uint32_t*>(so + tile * 512 + (jg & 31) * 16 + ((jg & 127) >> 5) * 4) = e8word;
     }
 }
 
@@ -202,7 +203,6 @@ __global__ void __launch_bounds__(128, 4) encode_b_kernel(const EncodeParams p)
     const int khalf = lane >> 4;
     const int kc = blockIdx.y;                      // chunk of 128 k
     const int b = blockIdx.z;
-    const int64_t qoff[4] = {0, (int64_t)p.cols, (int64_t)p.rows * p.ld, (int64_t)p.rows * p.ld + p.cols};
     const float* base = p.in + (int64_t)b * p.in_batch_stride + j;
     const int64_t term_codes = (int64_t)p.rows * p.cols;
 
@@ -223,7 +223,7 @@ __global__ void __launch_bounds__(128, 4) encode_b_kernel(const EncodeParams p)
                 if (jq < p.nq) {
 #pragma unroll
                     for (int kk = 0; kk < 16; ++kk)
-                        raw[jq][kk] = __ldg(base + qoff[jq] + (int64_t)(k0 + kk) * p.ld);
+                        raw[jq][kk] = __ldg(base + p.qoff[jq] + (int64_t)(k0 + kk) * p.ld);
                 }
 #pragma unroll
             for (int r = 0; r < FMM_MAX_RANK; ++r) {
@@ -266,7 +266,7 @@ __global__ void __launch_bounds__(128, 4) encode_b_kernel(const EncodeParams p)
                         blk_inv[r] = block_scale<MODE>(blk_amax[r], p.amax_floor, s, e8);
                         const int kb = (BLK == 32) ? (kc * 4 + sub) : kc;
                         e8word[r] |= e8 << (8 * (kb & 3));
-                        if (khalf == 0) store_b_scale<MODE>(p, t, j, kb, kc, s, e8word[r], (kb & 3) == 3);
+                        if (khalf == 0) store_b_scale<MODE>(p, t, r, j, kb, kc, s, e8word[r], (kb & 3) == 3);
                     }
                     if (BLK == 32 || pass == 1) {
                         const unsigned long long i2 = pack2(blk_inv[r], blk_inv[r]);

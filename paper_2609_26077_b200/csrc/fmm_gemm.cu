@@ -40,10 +40,6 @@ constexpr int REGS_AT_LAUNCH = 168, REGS_CTRL = 56, REGS_EPI = 224;
 static_assert(EPI_WARP0 * 32 * REGS_CTRL + EPI_WARPS * 32 * REGS_EPI <= NUM_THREADS * REGS_AT_LAUNCH, "register pool");
 static_assert(NUM_THREADS * (REGS_AT_LAUNCH + 8) > 65536, "REGS_AT_LAUNCH must be the launch-bound maximum");
 constexpr int STAGING_BYTES = 32 * 128; // 32 rows x 32 fp32 per epilogue warp and buffer
-#ifndef FMM_EXP_STAGING_BUFS
-#define FMM_EXP_STAGING_BUFS 2
-#endif
-constexpr int STAGING_BUFS = FMM_EXP_STAGING_BUFS;
 
 template <int BN, int MODE, int BLK, int NCTA>
 struct Cfg {
@@ -51,11 +47,10 @@ struct Cfg {
     static constexpr int BROWS = BN / NCTA;                  // T_r rows this CTA loads per stage
     static constexpr int A_BYTES = BM * BK;
     static constexpr int B_BYTES = BROWS * BK;
-#ifdef FMM_EXP_STAGES
-    static constexpr int STAGES = (NCTA == 2) ? FMM_EXP_STAGES : ((A_BYTES + B_BYTES) > 40000 ? 3 : 4);
-#else
-    static constexpr int STAGES = (A_BYTES + B_BYTES) > 40000 ? 3 : 4;
-#endif
+    // The UE8M0 pair kernel is bound by operand-load latency under L2 contention: it trades one
+    // epilogue staging buffer per warp for a fifth pipeline stage.
+    static constexpr int STAGING_BUFS = (MX && NCTA == 2) ? 1 : 2;
+    static constexpr int STAGES = (MX && NCTA == 2) ? 5 : ((A_BYTES + B_BYTES) > 40000 ? 3 : 4);
     static constexpr int SFB_ATOMS = BN / 128;
     static constexpr int SF_STAGE_BYTES = MX ? (512 + SFB_ATOMS * 512) : 0;
     static constexpr int KB_PER_STAGE = BK / BLK;
@@ -303,8 +298,8 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         const int e = warp - EPI_WARP0;
         const int q = warp & 3;            // TMEM lane quadrant this warp may access
         const int h = e >> 2;              // column half
-        const uint32_t stg = base + C::OFF_STG + e * STAGING_BUFS * STAGING_BYTES;
-        uint8_t* stg_ptr = base_ptr + C::OFF_STG + e * STAGING_BUFS * STAGING_BYTES;
+        const uint32_t stg = base + C::OFF_STG + e * C::STAGING_BUFS * STAGING_BYTES;
+        uint8_t* stg_ptr = base_ptr + C::OFF_STG + e * C::STAGING_BUFS * STAGING_BYTES;
         const uint32_t lane_taddr = tmem_base + ((uint32_t)(q * 32) << 16) + h * C::CW;
         // the accumulator-free signal goes to the MMA issuer, which lives in the even CTA
         auto release_acc = [&](int b) {
@@ -405,8 +400,8 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                     const int col0 = ent.col_off * p.n + tn * BN + h * C::CW;
 #pragma unroll
                     for (int c = 0; c < C::CW / 32; ++c) {
-                        const uint32_t b = store_cnt & (STAGING_BUFS - 1);
-                        if (lane == 0) bulk_wait_read<STAGING_BUFS - 1>();   // the buffer about to be rewritten has been read
+                        const uint32_t b = store_cnt & (C::STAGING_BUFS - 1);
+                        if (lane == 0) bulk_wait_read<C::STAGING_BUFS - 1>();   // the buffer about to be rewritten has been read
                         __syncwarp();
                         uint8_t* dst = stg_ptr + b * STAGING_BYTES + lane * 128;
 #pragma unroll

@@ -47,12 +47,16 @@ struct EncodeParams {
     int64_t ld;               // leading dimension of the input matrices
     int batch;                // number of input matrices
     int rows, cols;           // leaf (output) dimensions per combination
-    int nq;                   // 4: combine quadrants; 1: plain quantization of the matrix itself
+    int64_t qoff[4];          // element offsets of the four input blocks that are combined
+    int nq;                   // number of input blocks read (4, or 1 for a plain pass over one matrix)
     int R;                    // combinations per input matrix
     float coef[FMM_MAX_RANK][4];
     uint8_t* q_out;           // codes, term t = b * R + r at q_out + t * rows * cols
     void* s_out;              // scales
-    int64_t s_term_stride;    // bytes
+    int64_t s_term_stride;    // bytes between the scale arrays of consecutive terms
+    int s_step;               // rows (A side) / columns (B side) by which combination r is shifted inside a shared scale array
+    int s_ld;                 // B side, fp32 scales: row length of the scale array
+    int sf_blocks;            // UE8M0: number of 128-row blocks of the scale-tile array
     float amax_floor;
 };
 
