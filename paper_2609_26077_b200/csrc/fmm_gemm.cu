@@ -543,10 +543,18 @@ fmm_status_t launch(const GemmParams& g, cudaStream_t st)
 template <int MODE, int BLK>
 fmm_status_t launch_shape(const GemmParams& g, cudaStream_t st)
 {
-    // pairs of CTAs with 256 x 256 tiles whenever the leaf shape allows it; single CTAs otherwise
-    if ((g.m % 256) == 0 && (g.n % 256) == 0) return launch<256, MODE, BLK, 2>(g, st);
-    if ((g.n % 256) == 0) return launch<256, MODE, BLK, 1>(g, st);
-    return launch<128, MODE, BLK, 1>(g, st);
+    // Pairs of CTAs whenever the leaf shape allows it; single CTAs otherwise.  The UE8M0 kernel wants the
+    // widest tile (least operand traffic per MMA); the FP32-scale kernels are bound by the promotion
+    // on the CUDA cores and use 128-column tiles, whose four TMEM accumulators let the MMA issuer run
+    // further ahead of the promoting warps.
+    if constexpr (MODE != FMM_SCALE_UE8M0_CEIL) {
+        if ((g.m % 256) == 0) return launch<128, MODE, BLK, 2>(g, st);
+        return launch<128, MODE, BLK, 1>(g, st);
+    } else {
+        if ((g.m % 256) == 0 && (g.n % 256) == 0) return launch<256, MODE, 32, 2>(g, st);
+        if ((g.n % 256) == 0) return launch<256, MODE, 32, 1>(g, st);
+        return launch<128, MODE, 32, 1>(g, st);
+    }
 }
 
 }  // namespace
