@@ -1,0 +1,136 @@
+"""Error-measurement sweep on the GPU: relative Frobenius error of each realization against the fp64
+product, paired over identical operands and seeds, normalised by the cubic fp8 error (the paper's
+emulated protocol, App. E.2), for the benchmark configurations.
+
+    python -m paper_2609_26077_b200.sweep --config c1 [--scale-mode fp32|ue8m0] [--block-k 32|128]
+                                          [--out sweep.jsonl] [--trials N]
+    python -m paper_2609_26077_b200.sweep --summarise sweep.jsonl
+
+One JSON line is appended per (config, family, seed, realization, levels); on restart the keys that are
+already in the output file are skipped.  Everything is computed by the CUDA library (fmm_matmul,
+fmm_ref_gemm_fp64, fmm_error_stats); numpy only generates the seeded operands.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import sys
+from collections import defaultdict
+
+import numpy as np
+
+from . import fmm, realizations as P, workloads as Wl
+
+PREDICTED = {"cubic": 1.0, "strassen": 2.0, "winograd": math.sqrt(7.0), "phi_optimal": 5.0 / 3.0}
+ALL = ["cubic", "strassen", "winograd", "phi_optimal"]
+
+# name -> (M, K, N), families, trials, realizations, levels
+CONFIGS = {
+    "c1": dict(shape=(256, 256, 256), families=["gaussian"], trials=20, names=["cubic", "strassen"], levels=[1]),
+    "c2": dict(shape=(4096, 4096, 4096), families=["gaussian", "uniform"], trials=50, names=ALL, levels=[1]),
+    "c3": dict(shape=(8192, 8192, 8192), families=["gaussian"], trials=3, names=["cubic", "strassen", "phi_optimal"], levels=[1, 2]),
+    "c4": dict(shape=(16384, 8192, 8192), families=["llm"], trials=3, names=ALL, levels=[1]),
+    "c5": dict(shape=(2048, 2048, 2048), families=["scaled_gaussian", "student_t3"], trials=256, names=ALL, levels=[1, 2, 3]),
+}
+
+
+def _key(rec):
+    return (rec["config"], rec["family"], rec["seed"], rec["realization"], rec["levels"], rec["scale_mode"], rec["block_k"])
+
+
+def run(args):
+    import torch
+    cfg = CONFIGS[args.config]
+    M, K, N = cfg["shape"]
+    trials = args.trials or cfg["trials"]
+    done = set()
+    if os.path.exists(args.out):
+        for line in open(args.out):
+            try:
+                done.add(_key(json.loads(line)))
+            except Exception:
+                pass
+    plans = {}
+
+    def plan_for(name, lv):
+        k = (name, lv)
+        if k not in plans:
+            if name == "cubic":
+                plans[k] = fmm.Plan(levels=0, block_k=args.block_k, scale_mode=args.scale_mode)
+            else:
+                plans[k] = fmm.Plan(*P.get(name), levels=lv, block_k=args.block_k, scale_mode=args.scale_mode)
+        return plans[k]
+
+    out = open(args.out, "a")
+    C = torch.empty((M, N), dtype=torch.float32, device="cuda")
+    ref = torch.empty((M, N), dtype=torch.float64, device="cuda")
+    for family in cfg["families"]:
+        for seed in range(trials):
+            todo = [(n, lv) for n in cfg["names"] for lv in (cfg["levels"] if n != "cubic" else [0])
+                    if (args.config, family, seed, n, lv, args.scale_mode, args.block_k) not in done]
+            if not todo:
+                continue
+            A, B = Wl.FAMILIES[family](M, K, N, seed)
+            a, b = torch.from_numpy(A).cuda(), torch.from_numpy(B).cuda()
+            fmm.fmm_ref_gemm_fp64(a, b, out=ref)
+            for name, lv in todo:
+                pl = plan_for(name, lv)
+                pl.matmul(a, b, out=C)
+                s = fmm.fmm_error_stats(C, ref).cpu().numpy()
+                st, code = pl.device_status()
+                rec = {"config": args.config, "family": family, "seed": seed, "realization": name, "levels": lv,
+                       "scale_mode": args.scale_mode, "block_k": args.block_k, "M": M, "K": K, "N": N,
+                       "sum_sq_diff": float(s[0]), "sum_sq_ref": float(s[1]), "max_abs_diff": float(s[2]),
+                       "rel_frobenius": float(math.sqrt(s[0] / s[1])), "device_status": code}
+                out.write(json.dumps(rec) + "\n")
+                out.flush()
+            del a, b
+    out.close()
+
+
+def summarise(path, file=sys.stdout):
+    """Mean per-trial error, pooled RMS error and paired ratios vs cubic, per (config, family, levels)."""
+    recs = [json.loads(line) for line in open(path) if line.strip()]
+    groups = defaultdict(lambda: defaultdict(dict))
+    for r in recs:
+        g = (r["config"], r["family"], r["scale_mode"], r["block_k"])
+        groups[g][(r["realization"], r["levels"])][r["seed"]] = r
+    rows = []
+    for g, by in sorted(groups.items()):
+        cubic = by.get(("cubic", 0), {})
+        for (name, lv), seeds in sorted(by.items()):
+            e = np.array([seeds[s]["rel_frobenius"] for s in sorted(seeds)])
+            pooled = math.sqrt(sum(seeds[s]["sum_sq_diff"] for s in seeds) / sum(seeds[s]["sum_sq_ref"] for s in seeds))
+            common = [s for s in seeds if s in cubic]
+            ratio = (np.mean([seeds[s]["rel_frobenius"] for s in common]) /
+                     np.mean([cubic[s]["rel_frobenius"] for s in common])) if common else float("nan")
+            pred = PREDICTED.get(name, float("nan")) ** max(lv, 1) if name != "cubic" else 1.0
+            rows.append((g, name, lv, len(e), e.mean(), e.std(), pooled, ratio, pred))
+    print("| config | family | scales | blk | realization | levels | trials | mean rel. error | sd | pooled RMS | ratio vs cubic | sqrt(Phi/8)^l |", file=file)
+    print("|---|---|---|---|---|---|---|---|---|---|---|---|", file=file)
+    for g, name, lv, n, mean, sd, pooled, ratio, pred in rows:
+        print(f"| {g[0]} | {g[1]} | {g[2]} | {g[3]} | {name} | {lv} | {n} | {mean:.5f} | {sd:.5f} | {pooled:.5f} | {ratio:.4f} | {pred:.4f} |", file=file)
+    return rows
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--config", choices=sorted(CONFIGS))
+    ap.add_argument("--scale-mode", default="fp32", choices=["fp32", "ue8m0"])
+    ap.add_argument("--block-k", type=int, default=32, choices=[32, 128])
+    ap.add_argument("--out", default="sweep.jsonl")
+    ap.add_argument("--trials", type=int, default=0)
+    ap.add_argument("--summarise")
+    a = ap.parse_args()
+    if a.summarise:
+        summarise(a.summarise)
+    else:
+        if not a.config:
+            ap.error("--config or --summarise is required")
+        run(a)
+
+
+if __name__ == "__main__":
+    main()
