@@ -111,6 +111,21 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
+def reduce_max_ms(ms, dist=None, device="cpu"):
+    """Time of the slowest rank (replicas run independently; the job is as slow as its slowest replica)."""
+    if dist is None:
+        return ms
+    import torch
+    t = torch.tensor([ms], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def replica_throughput(flop_per_replica, world, ms_slowest):
+    """Whole-job value for `world` independent replicas timed by the slowest one, in TFLOP/s."""
+    return world * flop_per_replica / (ms_slowest * 1e-3) / 1e12
+
+
 def algorithmic_work(M, N, K, levels, rank, scale_bytes, blk):
     """Flops of the products and HBM bytes the method itself must move (fused post-addition):
     read A and B once, write then read the quantized operands and their scales once, write C once."""
@@ -169,12 +184,7 @@ def run_ours(args):
             fn()
         e1.record()
         barrier()
-        ms = e0.elapsed_time(e1)
-        if dist is not None:
-            t = torch.tensor([ms], device="cuda", dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
-        return ms / steps
+        return reduce_max_ms(e0.elapsed_time(e1), dist, "cuda") / steps
 
     plan = make_plan(args.realization, args.levels, args.block_k, args.scale_mode)
     ws = plan.workspace(M, N, K)
@@ -217,7 +227,7 @@ def run_ours(args):
     ms_e2e = time_steps(e2e_step, e2e_steps, 3)
 
     flop_eff = 2.0 * M * N * K
-    value = world * flop_eff / (ms_step * 1e-3) / 1e12
+    value = replica_throughput(flop_eff, world, ms_step)
     scale_bytes = 4 if args.scale_mode == "fp32" else 1
     rank_r = plan.rank if args.levels > 0 else 8
     flops_alg, enc_bytes, gemm_bytes = algorithmic_work(M, N, K, args.levels, rank_r, scale_bytes, args.block_k)
@@ -234,7 +244,7 @@ def run_ours(args):
                    "multi_gpu": "replicas only"},
         "clocks": clocks,
         "gpu_launches": launches_per_step * K_steps,
-        "e2e": {"value": world * flop_eff / (ms_e2e * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": ms_e2e,
+        "e2e": {"value": replica_throughput(flop_eff, world, ms_e2e), "unit": UNIT, "ms_per_step": ms_e2e,
                 "h2d_bytes_per_step": 4 * (M * K + K * N), "d2h_bytes_per_step": 4 * M * N, "steps": e2e_steps},
         "phases": {"encode_ms": enc_ms, "multiply_ms": mul_ms,
                    "encode_hbm_frac": enc_bytes / (enc_ms * 1e-3) / 1e9 / hbm,

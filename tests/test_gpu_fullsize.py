@@ -1,0 +1,48 @@
+"""GPU parity at the benchmark's full size (n = 8192, one level, Phi-optimal: the launch configuration
+bench.py times).  The quantized operands are compared in full against the oracle; C is compared on
+sampled rows that the oracle side computes one by one from its own quantized operands."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import oracle as O
+from paper_2609_26077_b200 import workloads as Wl
+from gpu_common import MODES, coeffs, dev, make_plan
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("mode,blk", [("fp32", 32), ("ue8m0", 32), ("fp32", 128)])
+def test_full_size_operands_bit_exact_and_sampled_rows_of_c(mode, blk):
+    n = 8192
+    h = n // 2
+    A, B = Wl.gaussian(n, n, n, seed=0)
+    plan = make_plan("phi_optimal", 1, blk, mode)
+    ws = plan.workspace(n, n, n)
+    C = plan.matmul(dev(A), dev(B), workspace=ws)
+    torch.cuda.synchronize()
+    assert plan.device_status() == (0, 0)
+    U, V, W = coeffs("phi_optimal")
+    ca, sa, ea = O.encode(A, "A", U, V, 1, blk, MODES[mode])
+    cb, sb, eb = O.encode(B, "B", U, V, 1, blk, MODES[mode])
+    rng = np.random.default_rng(1)
+    rows = np.sort(rng.choice(h, size=24, replace=False))
+    Mrows = []
+    for t in range(7):
+        qa, sca = plan.quantized_operand(ws, n, n, n, t, "A")
+        qb, scb = plan.quantized_operand(ws, n, n, n, t, "B")
+        assert np.array_equal(qa, ca[t]) and np.array_equal(qb, cb[t]), f"codes differ in term {t}"
+        assert np.array_equal(sca, sa[t] if mode == "fp32" else ea[t]), f"A scales differ in term {t}"
+        assert np.array_equal(scb, sb[t] if mode == "fp32" else eb[t]), f"B scales differ in term {t}"
+        # oracle side of the product for the sampled rows: exact dequantization, fp64 matmul
+        Sr = O.dequant_rows(ca[t][rows], sa[t][rows], blk)
+        Tr = O.dequant_cols(cb[t], sb[t], blk)
+        Mrows.append(Sr @ Tr)
+    got = C.cpu().numpy().astype(np.float64)
+    for q in range(4):
+        want = sum(float(W[r][q]) * Mrows[r] for r in range(7))
+        r0, c0 = (q >> 1) * h, (q & 1) * h
+        block = got[r0 + rows][:, c0:c0 + h]
+        rel = np.linalg.norm(block - want) / np.linalg.norm(want)
+        assert rel <= 1e-5, f"quadrant {q}: sampled rows differ by {rel:.3e}"
+    assert np.isfinite(got).all()
