@@ -72,20 +72,25 @@ __global__ void __launch_bounds__(256) encode_a_kernel(const EncodeParams p)
     constexpr int GROUP = BLK / 4;                 // lanes per block
     constexpr unsigned FULL = 0xffffffffu;
     const int lane = threadIdx.x & 31;
-    const int64_t warp_gid = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-    const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+    const uint32_t warp_gid = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const uint32_t nwarps = (gridDim.x * blockDim.x) >> 5;
     const int chunks = p.cols / 128;
     const int nkb = p.cols / BLK;
-    const int64_t units = (int64_t)p.batch * p.rows * chunks;
+    // a task is CPT consecutive 128-k chunks of one output row; tasks are dealt to warps round-robin
+    // (32-bit index arithmetic only: one division per task, none per chunk)
+    const int CPT = (chunks % 8 == 0) ? 8 : ((chunks % 4 == 0) ? 4 : 1);
+    const uint32_t tasks_per_row = (uint32_t)(chunks / CPT);
+    const uint32_t tasks = (uint32_t)p.batch * (uint32_t)p.rows * tasks_per_row;
     const int64_t term_codes = (int64_t)p.rows * p.cols;
     const bool b2 = lane & 4, b1 = lane & 2, b0 = lane & 1;
     const int my_r = lane & 7;
 
-    for (int64_t u = warp_gid; u < units; u += nwarps) {
-        const int c = (int)(u % chunks);
-        const int64_t bi = u / chunks;
-        const int i = (int)(bi % p.rows);
-        const int b = (int)(bi / p.rows);
+    for (uint32_t task = warp_gid; task < tasks; task += nwarps) {
+      const uint32_t row_id = task / tasks_per_row;
+      const int c0 = (int)(task - row_id * tasks_per_row) * CPT;
+      const int b = (int)(row_id / (uint32_t)p.rows);
+      const int i = (int)(row_id - (uint32_t)b * (uint32_t)p.rows);
+      for (int c = c0; c < c0 + CPT; ++c) {
         const float* base = p.in + (int64_t)b * p.in_batch_stride + (int64_t)i * p.ld + c * 128 + lane * 4;
         unsigned long long xl[4], xh[4];
 #pragma unroll
@@ -169,6 +174,7 @@ __global__ void __launch_bounds__(256) encode_a_kernel(const EncodeParams p)
                 *reinterpret_cast<uint32_t*>(so + tile * 512 + (ig & 31) * 16 + ((ig & 127) >> 5) * 4) = wv;
             }
         }
+      }
     }
 }
 
@@ -351,10 +357,12 @@ fmm_status_t fmm_launch_comb(const CombParams& p, cudaStream_t st)
 
 fmm_status_t fmm_launch_encode_a(const EncodeParams& p, int blk, int mode, cudaStream_t st)
 {
-    const int64_t units = (int64_t)p.batch * p.rows * (p.cols / 128);
-    int64_t blocks = (units + 7) / 8;
-    const int64_t cap = (int64_t)sm_count() * 8;
-    if (blocks > cap) blocks = cap;
+    // one task (8, 4 or 1 chunks of 128 k of one row) per warp; the block scheduler balances the SMs
+    const int chunks = p.cols / 128;
+    const int cpt = (chunks % 8 == 0) ? 8 : ((chunks % 4 == 0) ? 4 : 1);
+    const int64_t tasks = (int64_t)p.batch * p.rows * (chunks / cpt);
+    int64_t blocks = (tasks + 7) / 8;
+    if (blocks > 0x7fffffff) blocks = 0x7fffffff;
     const unsigned g = (unsigned)blocks;
     if (mode == FMM_SCALE_FP32_AMAX_DIV_448) {
         if (blk == 32) encode_a_kernel<32, FMM_SCALE_FP32_AMAX_DIV_448><<<g, 256, 0, st>>>(p);
