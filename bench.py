@@ -252,11 +252,17 @@ def run_ours(args):
                    "multiply_tflops": flops_alg / (mul_ms * 1e-3) / 1e12},
         "device_status": status[1],
     }
-    # dominant kernel = the tcgen05 product kernel
+    # dominant kernel = the tcgen05 product kernel.  DRAM traffic per launch: dram__bytes_read + write from the
+    # ncu capture at n = 4096 (profiles/fmm_gemm_kernel_n4096.md), scaled by the units processed (bytes ~ M*N)
+    measured_4096 = {("fp32", 32): 136.4e6, ("ue8m0", 32): 151.0e6}.get((args.scale_mode, args.block_k))
+    traffic = None
+    if measured_4096 is not None and args.levels == 1:
+        traffic = measured_4096 * (M * N) / (4096.0 * 4096.0)
     t_roof_ms = (flops_alg / (fp8_peak * 1e12) + (enc_bytes + gemm_bytes) / (hbm * 1e9)) * 1e3
     out["roofline"] = {"kernel": "fmm_gemm_kernel", "bound": "tensor",
                        "achieved": flops_alg / (mul_ms * 1e-3) / 1e12, "peak": fp8_peak, "unit": "TFLOP/s",
-                       "frac": flops_alg / (mul_ms * 1e-3) / 1e12 / fp8_peak, "traffic": None,
+                       "frac": flops_alg / (mul_ms * 1e-3) / 1e12 / fp8_peak, "traffic": traffic,
+                       "traffic_unit": "bytes per launch (ncu at n=4096, scaled)", "algorithmic_bytes": gemm_bytes,
                        "peak_source": f"2 x {pk['source']} bf16 burst ({pk['bf16_tflops']} TF/s)",
                        "combined_roofline_ms": t_roof_ms, "combined_frac": t_roof_ms / ms_step}
     if args.scale_mode == "fp32":
@@ -264,9 +270,15 @@ def run_ours(args):
         f = (rank_r / 8.0) ** args.levels if args.levels > 0 else 1.0
         lane_ops = 2.0 * M * N * (K / args.block_k) * f
         alu_peak = 148 * 128 * 1.965e9              # fp32 lanes x max SM clock, one op per lane per clock
-        out["roofline"].update({"bound": "alu" if lane_ops / alu_peak > flops_alg / (fp8_peak * 1e12) else "tensor",
-                                "alu_lane_ops": lane_ops, "alu_peak_lane_ops_per_s": alu_peak,
-                                "alu_frac": lane_ops / (mul_ms * 1e-3) / alu_peak})
+        t_alu, t_tc = lane_ops / alu_peak, flops_alg / (fp8_peak * 1e12)
+        t_roof_ms = (max(t_alu, t_tc) + (enc_bytes + gemm_bytes) / (hbm * 1e9)) * 1e3
+        r = out["roofline"]
+        r.update({"tensor_achieved_tflops": r["achieved"], "tensor_frac": r["frac"],
+                  "combined_roofline_ms": t_roof_ms, "combined_frac": t_roof_ms / ms_step})
+        if t_alu > t_tc:
+            r.update({"bound": "alu", "achieved": lane_ops / (mul_ms * 1e-3) / 1e12, "peak": alu_peak / 1e12,
+                      "unit": "T fp32 lane-op/s", "frac": lane_ops / (mul_ms * 1e-3) / alu_peak,
+                      "peak_source": "148 SMs x 128 fp32 lanes x 1.965 GHz (unit counts and max clock)"})
 
     if rank_id == 0 and world == 1 and not args.no_variants:
         variants = []
