@@ -67,7 +67,10 @@ struct Cfg {
     static constexpr int SMEM_BYTES = OFF_BAR + NUM_BARS * 8 + 16 + 1024;   // + alignment slack
     // TMEM: MX: one BN-column accumulator, then per stage 4 SFA + 4*(BN/128) SFB columns.
     //       FP32: ring of 512/BN accumulators, one per K block in flight.
-    static constexpr int ACC_BUFS = MX ? 1 : (512 / BN);
+    // FP32: GPB consecutive K blocks ("granules") share one completion signal: their MMAs are issued back to
+    // back into adjacent TMEM buffers and committed once, so the tensor pipe is not drained per K block.
+    static constexpr int GPB = MX ? 1 : ((KB_PER_STAGE >= 2 && 512 / BN >= 4) ? 2 : 1);
+    static constexpr int ACC_BUFS = MX ? 1 : (512 / BN) / GPB;        // ring of (GPB x BN)-column super-buffers
     static constexpr int SF_COLS = 4 + 4 * SFB_ATOMS;
     static constexpr int CW = BN / 2;      // columns per epilogue warp
     static_assert(SMEM_BYTES <= 232448, "shared memory budget");
@@ -94,7 +97,11 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const C
 {
     uint32_t spins = 0;
     uint64_t t0 = 0;
+#ifdef FMM_EXP_TEST_WAIT
+    while (!mbar_test_wait(bar, parity)) {
+#else
     while (!mbar_try_wait(bar, parity)) {
+#endif
         if ((++spins & 0x3FFu) == 0) {
             if (*ctl.abort_flag) return false;
             const uint64_t now = global_timer();
@@ -269,15 +276,18 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                             }
                         } else {
 #pragma unroll
-                            for (int g = 0; g < C::KB_PER_STAGE; ++g) {
+                            for (int g0 = 0; g0 < C::KB_PER_STAGE; g0 += C::GPB) {
                                 const long long tw3 = TCLK();
                                 if (!mbar_wait(bar_tempty(buf), bphase ^ 1u, ctl, 203)) { ok = false; break; }
                                 TADD(1, tw3);
                                 tc_fence_after();
 #pragma unroll
-                                for (int j = 0; j < BLK / 32; ++j) {
-                                    const int jj = g * (BLK / 32) + j;
-                                    mma_f8f6f4<NCTA>(tmem_base + buf * BN, adesc + 2 * jj, bdesc + 2 * jj, idesc, j > 0 ? 1u : 0u);
+                                for (int gi = 0; gi < C::GPB; ++gi) {
+#pragma unroll
+                                    for (int j = 0; j < BLK / 32; ++j) {
+                                        const int jj = (g0 + gi) * (BLK / 32) + j;
+                                        mma_f8f6f4<NCTA>(tmem_base + (buf * C::GPB + gi) * BN, adesc + 2 * jj, bdesc + 2 * jj, idesc, j > 0 ? 1u : 0u);
+                                    }
                                 }
                                 tc_commit<NCTA>(bar_tfull(buf));
                                 if (++buf == C::ACC_BUFS) { buf = 0; bphase ^= 1u; }
@@ -354,31 +364,35 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                         }
                         const uint8_t* sbs = base_ptr + C::OFF_SB + ss * C::SB_STAGE_BYTES;
 #pragma unroll
-                        for (int g = 0; g < C::KB_PER_STAGE; ++g) {
+                        for (int g0 = 0; g0 < C::KB_PER_STAGE; g0 += C::GPB) {
                             const long long tw = TCLK();
                             if (!mbar_wait_warp(bar_tfull(buf), bphase, ctl, 303)) { ok = false; break; }
                             TADD(3, tw);
                             tc_fence_after();
-                            const ulonglong2* sbg = reinterpret_cast<const ulonglong2*>(sbs + (g * BN + h * C::CW) * 4);
-                            const unsigned long long sa2 = pack2(sa[g], sa[g]);
-                            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + buf * BN + h * C::CW;
-                            uint32_t tmp[32];
 #pragma unroll
-                            for (int c = 0; c < C::CW / 32; ++c) {
-                                tmem_ld32(taddr + c * 32, tmp);      // a TMEM load round trip is a few tens of cycles
-                                tmem_ld_wait();
-                                if (c + 1 == C::CW / 32) {
-                                    // the last chunk is in registers: hand the TMEM buffer back before the arithmetic
-                                    tc_fence_before();
-                                    __syncwarp();
-                                    if (lane == 0) release_acc(buf);
-                                }
+                            for (int gi = 0; gi < C::GPB; ++gi) {
+                                const int g = g0 + gi;
+                                const ulonglong2* sbg = reinterpret_cast<const ulonglong2*>(sbs + (g * BN + h * C::CW) * 4);
+                                const unsigned long long sa2 = pack2(sa[g], sa[g]);
+                                const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (buf * C::GPB + gi) * BN + h * C::CW;
+                                uint32_t tmp[32];
 #pragma unroll
-                                for (int i = 0; i < 8; ++i) {
-                                    const ulonglong2 s4 = sbg[c * 8 + i];        // four column scales
-                                    const uint32_t* tp = tmp + 4 * i;
-                                    acc2[c * 16 + 2 * i] = fma2(pack2u(tp[0], tp[1]), mul2(sa2, s4.x), acc2[c * 16 + 2 * i]);
-                                    acc2[c * 16 + 2 * i + 1] = fma2(pack2u(tp[2], tp[3]), mul2(sa2, s4.y), acc2[c * 16 + 2 * i + 1]);
+                                for (int c = 0; c < C::CW / 32; ++c) {
+                                    tmem_ld32(taddr + c * 32, tmp);      // a TMEM load round trip is a few tens of cycles
+                                    tmem_ld_wait();
+                                    if (gi + 1 == C::GPB && c + 1 == C::CW / 32) {
+                                        // the last chunk is in registers: hand the TMEM buffers back before the arithmetic
+                                        tc_fence_before();
+                                        __syncwarp();
+                                        if (lane == 0) release_acc(buf);
+                                    }
+#pragma unroll
+                                    for (int i = 0; i < 8; ++i) {
+                                        const ulonglong2 s4 = sbg[c * 8 + i];        // four column scales
+                                        const uint32_t* tp = tmp + 4 * i;
+                                        acc2[c * 16 + 2 * i] = fma2(pack2u(tp[0], tp[1]), mul2(sa2, s4.x), acc2[c * 16 + 2 * i]);
+                                        acc2[c * 16 + 2 * i + 1] = fma2(pack2u(tp[2], tp[3]), mul2(sa2, s4.y), acc2[c * 16 + 2 * i + 1]);
+                                    }
                                 }
                             }
                             if (++buf == C::ACC_BUFS) { buf = 0; bphase ^= 1u; }
