@@ -66,7 +66,16 @@ __device__ __forceinline__ float block_scale(float amax, float floor_, float& s_
 // reduced with a transposing butterfly that leaves combination (lane & 7) in each lane, so the
 // two IEEE divisions of a block are executed once per block instead of once per lane and
 // combination; the multiplier is then broadcast back with one shuffle per combination.
-template <int BLK, int MODE>
+//
+// NZ is the zero pattern of the coefficients (bit 4r+j set when coef[r][j] != 0) when it is known at
+// compile time - the named realizations are pre-instantiated so that the zero tests, the "first term"
+// distinction and the rank guard cost nothing - or 0 for the generic run-time tests.
+template <uint32_t NZ> __device__ __forceinline__ bool coef_used(int r, int j, float c)
+{ return NZ ? ((NZ >> (4 * r + j)) & 1u) != 0 : (c != 0.0f); }
+template <uint32_t NZ> __device__ __forceinline__ bool row_used(int r, int R)
+{ return NZ ? ((NZ >> (4 * r)) & 15u) != 0 : (r < R); }
+
+template <int BLK, int MODE, uint32_t NZ>
 __global__ void __launch_bounds__(256) encode_a_kernel(const EncodeParams p)
 {
     constexpr int GROUP = BLK / 4;                 // lanes per block
@@ -92,33 +101,33 @@ __global__ void __launch_bounds__(256) encode_a_kernel(const EncodeParams p)
       const int i = (int)(row_id - (uint32_t)b * (uint32_t)p.rows);
       for (int c = c0; c < c0 + CPT; ++c) {
         const float* base = p.in + (int64_t)b * p.in_batch_stride + (int64_t)i * p.ld + c * 128 + lane * 4;
-        unsigned long long xl[4], xh[4];
+        float4 x[4];
 #pragma unroll
         for (int j = 0; j < 4; ++j)
-            if (j < p.nq) {
-                const float4 x = __ldcs(reinterpret_cast<const float4*>(base + p.qoff[j]));
-                xl[j] = pack2(x.x, x.y); xh[j] = pack2(x.z, x.w);
-            }
+            if (j < p.nq) x[j] = __ldcs(reinterpret_cast<const float4*>(base + p.qoff[j]));
 
-        unsigned long long vl[FMM_MAX_RANK], vh[FMM_MAX_RANK];
+        float4 v[FMM_MAX_RANK];
         float am[FMM_MAX_RANK];
 #pragma unroll
         for (int r = 0; r < FMM_MAX_RANK; ++r) {
-            vl[r] = 0ull; vh[r] = 0ull; am[r] = 0.0f;
-            if (r < p.R) {
+            v[r] = make_float4(0.f, 0.f, 0.f, 0.f); am[r] = 0.0f;
+            if (row_used<NZ>(r, p.R)) {
                 bool set = false;
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
                     const float cj = p.coef[r][j];
-                    if (cj != 0.0f) {
-                        const unsigned long long c2 = pack2(cj, cj);
-                        if (!set) { vl[r] = mul2(c2, xl[j]); vh[r] = mul2(c2, xh[j]); set = true; }
-                        else { vl[r] = fma2(c2, xl[j], vl[r]); vh[r] = fma2(c2, xh[j], vh[r]); }
+                    if (coef_used<NZ>(r, j, cj)) {
+                        if (!set) {
+                            v[r].x = __fmul_rn(cj, x[j].x); v[r].y = __fmul_rn(cj, x[j].y);
+                            v[r].z = __fmul_rn(cj, x[j].z); v[r].w = __fmul_rn(cj, x[j].w);
+                            set = true;
+                        } else {
+                            v[r].x = __fmaf_rn(cj, x[j].x, v[r].x); v[r].y = __fmaf_rn(cj, x[j].y, v[r].y);
+                            v[r].z = __fmaf_rn(cj, x[j].z, v[r].z); v[r].w = __fmaf_rn(cj, x[j].w, v[r].w);
+                        }
                     }
                 }
-                float a0, a1, a2, a3;
-                unpack2(vl[r], a0, a1); unpack2(vh[r], a2, a3);
-                am[r] = fmaxf(fmaxf(fabsf(a0), fabsf(a1)), fmaxf(fabsf(a2), fabsf(a3)));
+                am[r] = fmaxf(fmaxf(fabsf(v[r].x), fabsf(v[r].y)), fmaxf(fabsf(v[r].z), fabsf(v[r].w)));
             }
         }
         // transposing butterfly over the 8 lanes (lane & 7): afterwards `mine` is the maximum of
@@ -145,16 +154,15 @@ __global__ void __launch_bounds__(256) encode_a_kernel(const EncodeParams p)
         float s; uint32_t e8;
         const float inv = block_scale<MODE>(mine, p.amax_floor, s, e8);
 
-        uint8_t* qrow = p.q_out + ((int64_t)b * p.R) * term_codes + (int64_t)i * p.cols + c * 128 + lane * 4;
+        uint8_t* qp = p.q_out + ((int64_t)b * p.R) * term_codes + (int64_t)i * p.cols + c * 128 + lane * 4;
 #pragma unroll
         for (int r = 0; r < FMM_MAX_RANK; ++r) {
-            if (r < p.R) {
+            if (row_used<NZ>(r, p.R)) {
                 const float inv_r = __shfl_sync(FULL, inv, (GROUP == 32) ? r : ((lane & 24) | r));
-                const unsigned long long i2 = pack2(inv_r, inv_r);
-                float y0, y1, y2, y3;
-                unpack2(mul2(vl[r], i2), y0, y1); unpack2(mul2(vh[r], i2), y2, y3);
-                *reinterpret_cast<uint32_t*>(qrow + r * term_codes) = pack4_e4m3(y0, y1, y2, y3);
+                *reinterpret_cast<uint32_t*>(qp) = pack4_e4m3(__fmul_rn(v[r].x, inv_r), __fmul_rn(v[r].y, inv_r),
+                                                              __fmul_rn(v[r].z, inv_r), __fmul_rn(v[r].w, inv_r));
             }
+            qp += term_codes;
         }
         // scales: lane holds the scale of combination my_r, block (lane / GROUP) of this chunk
         if (MODE == FMM_SCALE_FP32_AMAX_DIV_448) {
@@ -199,7 +207,7 @@ __device__ __forceinline__ void store_b_scale(const EncodeParams& p, int64_t t, 
     }
 }
 
-template <int BLK, int MODE>
+template <int BLK, int MODE, uint32_t NZ>
 __global__ void __launch_bounds__(128, 4) encode_b_kernel(const EncodeParams p)
 {
     // here p.rows = leaf k (contracted), p.cols = leaf n
@@ -233,57 +241,49 @@ __global__ void __launch_bounds__(128, 4) encode_b_kernel(const EncodeParams p)
                 }
 #pragma unroll
             for (int r = 0; r < FMM_MAX_RANK; ++r) {
-                if (r < p.R) {
-                    unsigned long long v[8];
+                if (row_used<NZ>(r, p.R)) {
+                    float v[16];
                     bool set = false;
 #pragma unroll
                     for (int jq = 0; jq < 4; ++jq) {
                         const float cj = p.coef[r][jq];
-                        if (cj != 0.0f) {
-                            const unsigned long long c2 = pack2(cj, cj);
+                        if (coef_used<NZ>(r, jq, cj)) {
                             if (!set) {
 #pragma unroll
-                                for (int g = 0; g < 8; ++g) v[g] = mul2(c2, pack2(raw[jq][2 * g], raw[jq][2 * g + 1]));
+                                for (int kk = 0; kk < 16; ++kk) v[kk] = __fmul_rn(cj, raw[jq][kk]);
                                 set = true;
                             } else {
 #pragma unroll
-                                for (int g = 0; g < 8; ++g) v[g] = fma2(c2, pack2(raw[jq][2 * g], raw[jq][2 * g + 1]), v[g]);
+                                for (int kk = 0; kk < 16; ++kk) v[kk] = __fmaf_rn(cj, raw[jq][kk], v[kk]);
                             }
                         }
                     }
                     if (!set) {
 #pragma unroll
-                        for (int g = 0; g < 8; ++g) v[g] = 0ull;
+                        for (int kk = 0; kk < 16; ++kk) v[kk] = 0.0f;
                     }
                     const int64_t t = (int64_t)b * p.R + r;
                     if (BLK == 32 || pass == 0) {
                         float amax = 0.0f;
 #pragma unroll
-                        for (int g = 0; g < 8; ++g) {
-                            float a0, a1;
-                            unpack2(v[g], a0, a1);
-                            amax = fmaxf(amax, fmaxf(fabsf(a0), fabsf(a1)));
-                        }
+                        for (int kk = 0; kk < 16; ++kk) amax = fmaxf(amax, fabsf(v[kk]));
                         amax = fmaxf(amax, __shfl_xor_sync(FULL, amax, 16));
                         if (BLK == 32) blk_amax[r] = amax; else blk_amax[r] = fmaxf(blk_amax[r], amax);
                     }
                     if (BLK == 32 || (pass == 0 && sub == 3)) {
-                        float s; uint32_t e8;
-                        blk_inv[r] = block_scale<MODE>(blk_amax[r], p.amax_floor, s, e8);
+                        float sc; uint32_t e8;
+                        blk_inv[r] = block_scale<MODE>(blk_amax[r], p.amax_floor, sc, e8);
                         const int kb = (BLK == 32) ? (kc * 4 + sub) : kc;
                         e8word[r] |= e8 << (8 * (kb & 3));
-                        if (khalf == 0) store_b_scale<MODE>(p, t, r, j, kb, kc, s, e8word[r], (kb & 3) == 3);
+                        if (khalf == 0) store_b_scale<MODE>(p, t, r, j, kb, kc, sc, e8word[r], (kb & 3) == 3);
                     }
                     if (BLK == 32 || pass == 1) {
-                        const unsigned long long i2 = pack2(blk_inv[r], blk_inv[r]);
+                        const float inv = blk_inv[r];
                         uint32_t wv[4];
 #pragma unroll
-                        for (int g = 0; g < 4; ++g) {
-                            float y0, y1, y2, y3;
-                            unpack2(mul2(v[2 * g], i2), y0, y1);
-                            unpack2(mul2(v[2 * g + 1], i2), y2, y3);
-                            wv[g] = pack4_e4m3(y0, y1, y2, y3);
-                        }
+                        for (int g = 0; g < 4; ++g)
+                            wv[g] = pack4_e4m3(__fmul_rn(v[4 * g], inv), __fmul_rn(v[4 * g + 1], inv),
+                                               __fmul_rn(v[4 * g + 2], inv), __fmul_rn(v[4 * g + 3], inv));
                         *reinterpret_cast<uint4*>(p.q_out + t * term_codes + (int64_t)j * p.rows + k0) =
                             make_uint4(wv[0], wv[1], wv[2], wv[3]);
                     }
@@ -355,6 +355,44 @@ fmm_status_t fmm_launch_comb(const CombParams& p, cudaStream_t st)
     return cudaGetLastError() == cudaSuccess ? FMM_OK : FMM_ERR_CUDA;
 }
 
+namespace {
+uint32_t coef_mask(const EncodeParams& p)
+{
+    uint32_t m = 0;
+    for (int r = 0; r < p.R; ++r)
+        for (int j = 0; j < 4; ++j)
+            if (p.coef[r][j] != 0.0f) m |= 1u << (4 * r + j);
+    return m;
+}
+
+// zero patterns with pre-instantiated kernels: U and V of Strassen, the Winograd form and the
+// Phi-optimal realization, and the identity used to quantize a matrix as four panels
+#define FMM_KNOWN_MASKS(X) X(0x0a5381c9u) X(0x0c385a19u) X(0x05dc8f21u) X(0x0ab3f841u) X(0x0f5fc5c9u) X(0x0cfc5f59u) X(0x00008421u)
+
+template <int BLK, int MODE>
+void launch_a(const EncodeParams& p, unsigned g, cudaStream_t st)
+{
+    const uint32_t m = (p.nq == 4) ? coef_mask(p) : 0u;
+    switch (m) {
+#define X(M) case M: encode_a_kernel<BLK, MODE, M><<<g, 256, 0, st>>>(p); return;
+        FMM_KNOWN_MASKS(X)
+#undef X
+        default: encode_a_kernel<BLK, MODE, 0u><<<g, 256, 0, st>>>(p); return;
+    }
+}
+template <int BLK, int MODE>
+void launch_b(const EncodeParams& p, dim3 grid, cudaStream_t st)
+{
+    const uint32_t m = (p.nq == 4) ? coef_mask(p) : 0u;
+    switch (m) {
+#define X(M) case M: encode_b_kernel<BLK, MODE, M><<<grid, 128, 0, st>>>(p); return;
+        FMM_KNOWN_MASKS(X)
+#undef X
+        default: encode_b_kernel<BLK, MODE, 0u><<<grid, 128, 0, st>>>(p); return;
+    }
+}
+}  // namespace
+
 fmm_status_t fmm_launch_encode_a(const EncodeParams& p, int blk, int mode, cudaStream_t st)
 {
     // one task (8, 4 or 1 chunks of 128 k of one row) per warp; the block scheduler balances the SMs
@@ -365,10 +403,10 @@ fmm_status_t fmm_launch_encode_a(const EncodeParams& p, int blk, int mode, cudaS
     if (blocks > 0x7fffffff) blocks = 0x7fffffff;
     const unsigned g = (unsigned)blocks;
     if (mode == FMM_SCALE_FP32_AMAX_DIV_448) {
-        if (blk == 32) encode_a_kernel<32, FMM_SCALE_FP32_AMAX_DIV_448><<<g, 256, 0, st>>>(p);
-        else encode_a_kernel<128, FMM_SCALE_FP32_AMAX_DIV_448><<<g, 256, 0, st>>>(p);
+        if (blk == 32) launch_a<32, FMM_SCALE_FP32_AMAX_DIV_448>(p, g, st);
+        else launch_a<128, FMM_SCALE_FP32_AMAX_DIV_448>(p, g, st);
     } else {
-        encode_a_kernel<32, FMM_SCALE_UE8M0_CEIL><<<g, 256, 0, st>>>(p);
+        launch_a<32, FMM_SCALE_UE8M0_CEIL>(p, g, st);
     }
     return cudaGetLastError() == cudaSuccess ? FMM_OK : FMM_ERR_CUDA;
 }
@@ -377,10 +415,10 @@ fmm_status_t fmm_launch_encode_b(const EncodeParams& p, int blk, int mode, cudaS
 {
     dim3 grid((unsigned)(p.cols / 64), (unsigned)(p.rows / 128), (unsigned)p.batch);
     if (mode == FMM_SCALE_FP32_AMAX_DIV_448) {
-        if (blk == 32) encode_b_kernel<32, FMM_SCALE_FP32_AMAX_DIV_448><<<grid, 128, 0, st>>>(p);
-        else encode_b_kernel<128, FMM_SCALE_FP32_AMAX_DIV_448><<<grid, 128, 0, st>>>(p);
+        if (blk == 32) launch_b<32, FMM_SCALE_FP32_AMAX_DIV_448>(p, grid, st);
+        else launch_b<128, FMM_SCALE_FP32_AMAX_DIV_448>(p, grid, st);
     } else {
-        encode_b_kernel<32, FMM_SCALE_UE8M0_CEIL><<<grid, 128, 0, st>>>(p);
+        launch_b<32, FMM_SCALE_UE8M0_CEIL>(p, grid, st);
     }
     return cudaGetLastError() == cudaSuccess ? FMM_OK : FMM_ERR_CUDA;
 }
