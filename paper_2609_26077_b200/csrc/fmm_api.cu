@@ -60,13 +60,14 @@ void make_layout(const fmm_plan* plan, int64_t M, int64_t N, int64_t K, FmmLayou
     L->sb_term = (size_t)(L->n * nkb) * sbytes;
     L->sa = off; off = align_up(off + L->sa_term * L->terms, 1024);
     L->sb = off; off = align_up(off + L->sb_term * L->terms, 1024);
-    for (int lv = 0; lv < FMM_MAX_LEVELS; ++lv) { L->inter_a[lv] = 0; L->inter_b[lv] = 0; }
+    for (int lv = 0; lv < FMM_MAX_LEVELS; ++lv) { L->inter_a[lv] = 0; L->inter_b[lv] = 0; L->dec[lv] = 0; }
     // fp32 combinations of the outer levels 1 .. levels-1
     for (int lv = 1; lv < plan->levels; ++lv) {
         const int64_t cnt = fmm_ipow(plan->rank, lv);
         const int64_t dd = (int64_t)1 << lv;
         L->inter_a[lv] = off; off = align_up(off + (size_t)(cnt * (M / dd) * (K / dd)) * 4, 1024);
         L->inter_b[lv] = off; off = align_up(off + (size_t)(cnt * (K / dd) * (N / dd)) * 4, 1024);
+        L->dec[lv] = off; off = align_up(off + (size_t)(cnt * (M / dd) * (N / dd)) * 4, 1024);
     }
     L->total = off;
 }
@@ -167,13 +168,36 @@ fmm_status_t multiply(fmm_plan* plan, const FmmLayout& L, char* ws, float* C, in
     g.qb = reinterpret_cast<const uint8_t*>(ws + L.qb);
     g.sa = ws + L.sa; g.sb = ws + L.sb;
     g.sa_term = (int64_t)L.sa_term; g.sb_term = (int64_t)L.sb_term;
-    g.C = C; g.ldc = N; g.Mfull = M; g.Nfull = N;
+    // The product kernel applies the innermost decoder only: leaf products of parent p land in the four
+    // blocks of parent p's (2m x 2n) matrix.  For one level that matrix is C itself; for more levels the
+    // parents' matrices are stacked in the workspace and decoded outwards level by level (the same
+    // two-stage order as the recursion in Sec. 3), which moves far fewer bytes than scattering every
+    // leaf product into all of its R^(levels-1)-fold weighted destinations.
+    const int lv = plan->levels;
+    const int64_t parents = lv >= 2 ? fmm_ipow(plan->rank, lv - 1) : 1;
+    const int64_t pm = lv >= 1 ? 2 * L.m : L.m, pn = lv >= 1 ? 2 * L.n : L.n;      // a parent's matrix
+    float* dest = lv >= 2 ? reinterpret_cast<float*>(ws + L.dec[lv - 1]) : C;
+    g.C = dest; g.ldc = pn; g.Mfull = parents * pm; g.Nfull = pn;
     g.m = (int)L.m; g.n = (int)L.n; g.k = (int)L.k; g.terms = (int)L.terms;
     g.out_start = plan->d_out_start; g.out = plan->d_out; g.status = plan->d_status;
     int launches = 0;
     fmm_status_t s = fmm_launch_gemm(g, plan->qp.block_k, (int)plan->qp.scale_mode, st, &launches);
     plan->last_launches += launches;
-    return s;
+    if (s != FMM_OK) return s;
+    for (int l = lv - 1; l >= 1; --l) {
+        DecodeParams d;
+        memset(&d, 0, sizeof(d));
+        d.in = reinterpret_cast<const float*>(ws + L.dec[l]);
+        d.out = l == 1 ? C : reinterpret_cast<float*>(ws + L.dec[l - 1]);
+        d.batch = (int)fmm_ipow(plan->rank, l - 1);
+        d.rows = (int)(M >> l); d.cols = (int)(N >> l); d.R = plan->rank;
+        for (int r = 0; r < plan->rank; ++r)
+            for (int q = 0; q < 4; ++q) d.W[r][q] = plan->W[r][q];
+        s = fmm_launch_decode(d, st);
+        if (s != FMM_OK) return s;
+        plan->last_launches++;
+    }
+    return FMM_OK;
 }
 
 }  // namespace
@@ -253,32 +277,28 @@ fmm_status_t fmm_plan_create(fmm_plan_t** out, int rank, const float* U, const f
             for (int j = 0; j < 4; ++j) { p->U[r][j] = U[r * 4 + j]; p->V[r][j] = V[r * 4 + j]; p->W[r][j] = W[r * 4 + j]; }
     p->terms = (int)fmm_ipow(rank, levels);
 
-    // Decoder table: destinations of every leaf product (Sec. 2.1 decode; Kronecker power for levels > 1).
-    const int nb = 1 << levels;                       // leaf blocks per side of C
+    // Decoder table of the product kernel: leaf product t = parent * R + r goes to block q of its parent's
+    // matrix with weight W[r][q] (Sec. 2.1 decode, innermost level; outer levels are decoded afterwards).
+    // row_off / col_off are in units of leaf blocks inside the stack of parent matrices.
     std::vector<int> start(p->terms + 1, 0);
     std::vector<FmmOutEntry> entries;
-    std::vector<char> touched((size_t)nb * nb, 0);
+    const int parents = levels >= 1 ? p->terms / rank : 1;
+    std::vector<char> touched((size_t)parents * 4, 0);
     for (int t = 0; t < p->terms; ++t) {
         start[t] = (int)entries.size();
-        int digits[FMM_MAX_LEVELS] = {0, 0, 0};
-        int tt = t;
-        for (int l = levels - 1; l >= 0; --l) { digits[l] = tt % rank; tt /= rank; }
-        const int paths = 1 << (2 * levels);
-        for (int path = 0; path < paths; ++path) {
-            double w = 1.0;
-            int rb = 0, cb = 0;
-            for (int l = 0; l < levels; ++l) {
-                const int q = (path >> (2 * (levels - 1 - l))) & 3;
-                w *= (double)p->W[digits[l]][q];
-                rb = rb * 2 + (q >> 1);
-                cb = cb * 2 + (q & 1);
-            }
-            if (levels == 0) { w = 1.0; }
-            if (w == 0.0) continue;
+        if (levels == 0) {
+            FmmOutEntry e; e.row_off = 0; e.col_off = 0; e.w = 1.0f; e.first = 1;
+            entries.push_back(e);
+            continue;
+        }
+        const int parent = t / rank, r = t % rank;
+        for (int q = 0; q < 4; ++q) {
+            const float w = p->W[r][q];
+            if (w == 0.0f) continue;
             FmmOutEntry e;
-            e.row_off = rb; e.col_off = cb; e.w = (float)w;
-            e.first = touched[(size_t)rb * nb + cb] ? 0 : 1;
-            touched[(size_t)rb * nb + cb] = 1;
+            e.row_off = parent * 2 + (q >> 1); e.col_off = q & 1; e.w = w;
+            e.first = touched[(size_t)parent * 4 + q] ? 0 : 1;
+            touched[(size_t)parent * 4 + q] = 1;
             entries.push_back(e);
         }
     }

@@ -331,6 +331,49 @@ __global__ void __launch_bounds__(256) comb_kernel(const CombParams p)
     }
 }
 
+// Outward step of the decoder for levels >= 2: the R partially decoded products of a parent are
+// combined into the four blocks of the parent's matrix, out_q = sum_r W[r][q] * in_r (fp32, r ascending,
+// zero weights skipped, first term a multiply, later terms FMAs).
+__global__ void __launch_bounds__(256) decode_kernel(const DecodeParams p)
+{
+    const int c4 = p.cols / 4;
+    const int64_t units = (int64_t)p.batch * p.rows * c4;
+    const int64_t in_stride = (int64_t)p.rows * p.cols;
+    const int64_t out_ld = 2 * (int64_t)p.cols;
+    for (int64_t u = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; u < units; u += (int64_t)gridDim.x * blockDim.x) {
+        const int c = (int)(u % c4);
+        const int64_t bi = u / c4;
+        const int i = (int)(bi % p.rows);
+        const int b = (int)(bi / p.rows);
+        float4 acc[4];
+        bool set[4] = {false, false, false, false};
+#pragma unroll
+        for (int q = 0; q < 4; ++q) acc[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+        const float* src = p.in + ((int64_t)b * p.R) * in_stride + (int64_t)i * p.cols + c * 4;
+        for (int r = 0; r < p.R; ++r) {
+            const float4 x = __ldcs(reinterpret_cast<const float4*>(src + r * in_stride));
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const float w = p.W[r][q];
+                if (w != 0.0f) {
+                    if (!set[q]) {
+                        acc[q].x = __fmul_rn(w, x.x); acc[q].y = __fmul_rn(w, x.y);
+                        acc[q].z = __fmul_rn(w, x.z); acc[q].w = __fmul_rn(w, x.w);
+                        set[q] = true;
+                    } else {
+                        acc[q].x = __fmaf_rn(w, x.x, acc[q].x); acc[q].y = __fmaf_rn(w, x.y, acc[q].y);
+                        acc[q].z = __fmaf_rn(w, x.z, acc[q].z); acc[q].w = __fmaf_rn(w, x.w, acc[q].w);
+                    }
+                }
+            }
+        }
+        float* dst = p.out + (int64_t)b * 4 * in_stride;
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+            *reinterpret_cast<float4*>(dst + ((int64_t)(q >> 1) * p.rows + i) * out_ld + (q & 1) * p.cols + c * 4) = acc[q];
+    }
+}
+
 int sm_count()
 {
     static int n = 0;
@@ -344,6 +387,16 @@ int sm_count()
 }
 
 }  // namespace
+
+fmm_status_t fmm_launch_decode(const DecodeParams& p, cudaStream_t st)
+{
+    const int64_t units = (int64_t)p.batch * p.rows * (p.cols / 4);
+    int64_t blocks = (units + 255) / 256;
+    const int64_t cap = (int64_t)sm_count() * 16;
+    if (blocks > cap) blocks = cap;
+    decode_kernel<<<(unsigned)blocks, 256, 0, st>>>(p);
+    return cudaGetLastError() == cudaSuccess ? FMM_OK : FMM_ERR_CUDA;
+}
 
 fmm_status_t fmm_launch_comb(const CombParams& p, cudaStream_t st)
 {

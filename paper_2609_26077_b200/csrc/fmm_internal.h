@@ -24,6 +24,7 @@ struct FmmLayout {            // byte offsets into the workspace
     size_t sa, sb;            // scales
     size_t sa_term, sb_term;  // bytes of scales per term
     size_t inter_a[FMM_MAX_LEVELS], inter_b[FMM_MAX_LEVELS];  // fp32 combinations of outer levels
+    size_t dec[FMM_MAX_LEVELS];   // dec[l]: R^l partially decoded products of (M/2^l) x (N/2^l) fp32, l = 1 .. levels-1
     size_t total;
 };
 
@@ -68,6 +69,14 @@ struct CombParams {
     float* out;               // dense rows x cols per (b, r)
 };
 
+// One outward step of the decoder: out[b] (2*rows x 2*cols, block q at (q>>1, q&1)) = sum_r W[r][q] * in[b*R + r]
+struct DecodeParams {
+    const float* in;          // batch * R matrices, rows x cols each, dense
+    float* out;               // batch matrices, 2*rows x 2*cols each, dense
+    int batch, rows, cols, R;
+    float W[FMM_MAX_RANK][4];
+};
+fmm_status_t fmm_launch_decode(const DecodeParams& p, cudaStream_t st);
 fmm_status_t fmm_launch_comb(const CombParams& p, cudaStream_t st);
 fmm_status_t fmm_launch_encode_a(const EncodeParams& p, int blk, int mode, cudaStream_t st);
 fmm_status_t fmm_launch_encode_b(const EncodeParams& p, int blk, int mode, cudaStream_t st);
