@@ -82,7 +82,7 @@ fmm_status_t fmm_plan_destroy(fmm_plan_t* plan);
 
 /* Bytes of device workspace fmm_matmul / fmm_encode_only need for this problem size (host call).
  * The workspace holds the quantized leaf operands, their scales and, for levels >= 2, the fp32
- * intermediate combinations of the outer levels. */
+ * intermediate combinations of the outer levels and the partially decoded products. */
 fmm_status_t fmm_workspace_bytes(const fmm_plan_t* plan, int64_t M, int64_t N, int64_t K,
                                  size_t* bytes);
 

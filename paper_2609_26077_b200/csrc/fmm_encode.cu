@@ -99,12 +99,21 @@ __global__ void __launch_bounds__(256) encode_a_kernel(const EncodeParams p)
       const int c0 = (int)(task - row_id * tasks_per_row) * CPT;
       const int b = (int)(row_id / (uint32_t)p.rows);
       const int i = (int)(row_id - (uint32_t)b * (uint32_t)p.rows);
+      // the loads of chunk c+1 are issued before chunk c is processed (two chunks in flight per warp)
+      const float* row_base = p.in + (int64_t)b * p.in_batch_stride + (int64_t)i * p.ld + lane * 4;
+      float4 xn[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j)
+          if (j < p.nq) xn[j] = __ldcs(reinterpret_cast<const float4*>(row_base + c0 * 128 + p.qoff[j]));
       for (int c = c0; c < c0 + CPT; ++c) {
-        const float* base = p.in + (int64_t)b * p.in_batch_stride + (int64_t)i * p.ld + c * 128 + lane * 4;
         float4 x[4];
 #pragma unroll
-        for (int j = 0; j < 4; ++j)
-            if (j < p.nq) x[j] = __ldcs(reinterpret_cast<const float4*>(base + p.qoff[j]));
+        for (int j = 0; j < 4; ++j) x[j] = xn[j];
+        if (c + 1 < c0 + CPT) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                if (j < p.nq) xn[j] = __ldcs(reinterpret_cast<const float4*>(row_base + (c + 1) * 128 + p.qoff[j]));
+        }
 
         float4 v[FMM_MAX_RANK];
         float am[FMM_MAX_RANK];
