@@ -158,6 +158,16 @@ int64_t fmm_error_stats_noalloc_max_elements(void);
  * call that set it are invalid.  Returns FMM_ERR_DEVICE_TIMEOUT when *code != 0. */
 fmm_status_t fmm_device_status(const fmm_plan_t* plan, int* code);
 
+/* Resets the plan's status words to zero (synchronises the device). */
+fmm_status_t fmm_device_status_clear(const fmm_plan_t* plan);
+
+/* Self-test of the failure-detection path (no counterpart in the paper): enqueues a one-warp kernel that
+ * waits, with the library's bounded-wait routine, on a barrier that nothing signals.  After limit_ns
+ * (1 .. 2e9 nanoseconds) the wait gives up, writes location code 901 into the status word and the kernel
+ * ends normally - the context stays usable.  fmm_device_status then reports FMM_ERR_DEVICE_TIMEOUT until
+ * fmm_device_status_clear is called. */
+fmm_status_t fmm_selftest_bounded_wait(const fmm_plan_t* plan, int64_t limit_ns, void* cuda_stream);
+
 /* Host utility (Sec. 2.1): Phi = sum_r |U_r|^2 |V_r|^2 |W_r|^2 and Gamma = sum_r |U_r| |V_r| |W_r|
  * with entrywise 2-norms, in fp64. */
 fmm_status_t fmm_phi_gamma(int rank, const float* U, const float* V, const float* W,

@@ -427,6 +427,19 @@ fmm_status_t fmm_debug_status64(const fmm_plan_t* plan, int* out64)
 }
 #endif
 
+fmm_status_t fmm_device_status_clear(const fmm_plan_t* plan)
+{
+    if (!plan) return FMM_ERR_INVALID_ARG;
+    if (cudaMemset(plan->d_status, 0, 64 * sizeof(int)) != cudaSuccess) { cudaGetLastError(); return FMM_ERR_CUDA; }
+    return FMM_OK;
+}
+
+fmm_status_t fmm_selftest_bounded_wait(const fmm_plan_t* plan, int64_t limit_ns, void* stream)
+{
+    if (!plan || limit_ns <= 0 || limit_ns > 2000000000ll) return FMM_ERR_INVALID_ARG;
+    return fmm_launch_bounded_wait_selftest(plan->d_status, (unsigned long long)limit_ns, reinterpret_cast<cudaStream_t>(stream));
+}
+
 fmm_status_t fmm_last_launch_count(const fmm_plan_t* plan, int* launches)
 {
     if (!plan || !launches) return FMM_ERR_INVALID_ARG;

@@ -90,6 +90,7 @@ constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;   // 2 s: far beyond
 struct Ctl {
     volatile int* abort_flag;   // shared memory
     int* status;                // global status words
+    unsigned long long limit_ns = WAIT_LIMIT_NS;
 };
 
 // Bounded mbarrier wait.  Returns false after WAIT_LIMIT_NS or when another role has given up.
@@ -106,7 +107,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const C
             if (*ctl.abort_flag) return false;
             const uint64_t now = global_timer();
             if (t0 == 0) t0 = now;
-            else if (now - t0 > WAIT_LIMIT_NS) {
+            else if (now - t0 > ctl.limit_ns) {
                 *ctl.abort_flag = 1;
                 atomicCAS(ctl.status, 0, where);
                 return false;
@@ -120,6 +121,19 @@ __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, co
 {
     const bool ok = mbar_wait(bar, parity, ctl, where);
     return __all_sync(0xffffffffu, ok);
+}
+
+// Self-test of the bounded wait: one warp waits on a barrier that nothing ever signals; the wait must
+// give up after limit_ns, record `where` in the status word and let the kernel end normally.
+__global__ void bounded_wait_selftest_kernel(int* status, unsigned long long limit_ns, int where)
+{
+    __shared__ __align__(8) unsigned long long bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) { mbar_init(smem_u32(&bar), 1); abort_flag = 0; fence_barrier_init(); }
+    __syncthreads();
+    Ctl ctl{&abort_flag, status, limit_ns};
+    const bool ok = mbar_wait_warp(smem_u32(&bar), 0, ctl, where);
+    if (threadIdx.x == 0 && ok) atomicExch(status + 1, 1);      // must not happen: nothing arrives on the barrier
 }
 
 struct KParams {
@@ -572,6 +586,12 @@ fmm_status_t launch_shape(const GemmParams& g, cudaStream_t st)
 }
 
 }  // namespace
+
+fmm_status_t fmm_launch_bounded_wait_selftest(int* status, unsigned long long limit_ns, cudaStream_t st)
+{
+    bounded_wait_selftest_kernel<<<1, 32, 0, st>>>(status, limit_ns, 901);
+    return cudaGetLastError() == cudaSuccess ? FMM_OK : FMM_ERR_CUDA;
+}
 
 fmm_status_t fmm_launch_gemm(const GemmParams& g, int blk, int mode, cudaStream_t st, int* launches)
 {

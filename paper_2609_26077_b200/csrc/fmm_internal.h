@@ -91,6 +91,7 @@ struct GemmParams {
     const int* out_start; const FmmOutEntry* out;
     int* status;
 };
+fmm_status_t fmm_launch_bounded_wait_selftest(int* status, unsigned long long limit_ns, cudaStream_t st);
 fmm_status_t fmm_launch_gemm(const GemmParams& p, int blk, int mode, cudaStream_t st, int* launches);
 
 static inline int64_t fmm_ipow(int64_t b, int e) { int64_t r = 1; while (e-- > 0) r *= b; return r; }

@@ -19,7 +19,7 @@ SCALE_MODES = {"fp32": SCALE_FP32, "ue8m0": SCALE_UE8M0}
 EXPORTS = ["fmm_plan_create", "fmm_plan_destroy", "fmm_workspace_bytes", "fmm_matmul", "fmm_encode_only",
            "fmm_multiply_only", "fmm_quantized_view", "fmm_ref_gemm_fp64", "fmm_error_stats",
            "fmm_error_stats_scratch_bytes", "fmm_error_stats_noalloc", "fmm_error_stats_noalloc_max_elements",
-           "fmm_device_status", "fmm_phi_gamma", "fmm_brent_residual",
+           "fmm_device_status", "fmm_device_status_clear", "fmm_selftest_bounded_wait", "fmm_phi_gamma", "fmm_brent_residual",
            "fmm_last_launch_count", "fmm_status_string"]
 
 
@@ -199,6 +199,13 @@ class Plan:
         code = C.c_int()
         st = lib().fmm_device_status(self._h, C.byref(code))
         return st, code.value
+
+    def device_status_clear(self):
+        _check(lib().fmm_device_status_clear(self._h), "fmm_device_status_clear")
+
+    def selftest_bounded_wait(self, limit_ns, stream=None):
+        _check(lib().fmm_selftest_bounded_wait(self._h, C.c_int64(int(limit_ns)), _stream_ptr(stream)),
+               "fmm_selftest_bounded_wait")
 
     def last_launch_count(self):
         n = C.c_int()

@@ -1,0 +1,94 @@
+"""GPU checks of the boundary's error behaviour, of properties that hold at any size, and of the
+bounded-wait failure path (a wait that runs out must leave a status code and a usable context)."""
+import ctypes as C
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import oracle as O
+from paper_2609_26077_b200 import fmm, realizations as P, workloads as Wl
+from gpu_common import dev, make_plan
+
+pytestmark = pytest.mark.gpu
+
+
+def test_matmul_rejects_bad_shapes_workspace_and_pointers():
+    plan = make_plan("strassen", 1, 32, "fp32")
+    lib = fmm.lib()
+    a = torch.zeros(256, 256, device="cuda")
+    c = torch.zeros(256, 256, device="cuda")
+    ws = plan.workspace(256, 256, 256)
+    p = lambda t: C.c_void_p(t.data_ptr())
+    call = lambda M, N, K, w, wb, A=a, B=a, Cc=c: lib.fmm_matmul(plan._h, p(A) if A is not None else None, p(B), p(Cc),
+                                                                 C.c_int64(M), C.c_int64(N), C.c_int64(K), w, C.c_size_t(wb), None)
+    assert call(256, 256, 256, p(ws), ws.numel()) == 0
+    assert call(192, 256, 256, p(ws), ws.numel()) == 2          # M/2 not a multiple of 128
+    assert call(256, 256, 320, p(ws), ws.numel()) == 2          # K/2 not a multiple of 128
+    assert call(0, 256, 256, p(ws), ws.numel()) == 2
+    assert call(256, 256, 256, p(ws), ws.numel() - 1) == 4      # workspace too small
+    assert call(256, 256, 256, None, ws.numel()) == 4
+    assert call(256, 256, 256, C.c_void_p(ws.data_ptr() + 8), ws.numel()) == 4   # misaligned
+    assert call(256, 256, 256, p(ws), ws.numel(), A=None) == 1
+    need = C.c_size_t()
+    assert lib.fmm_workspace_bytes(plan._h, C.c_int64(100), C.c_int64(256), C.c_int64(256), C.byref(need)) == 2
+    torch.cuda.synchronize()
+    assert plan.device_status() == (0, 0)
+
+
+def test_power_of_two_rescaling_leaves_codes_identical_on_device():
+    # App. E.2: Q(2^k x) has the same codes and 2^k-times the scales
+    A, B = Wl.gaussian(256, 256, 256, 4)
+    plan = make_plan("phi_optimal", 1, 32, "fp32")
+    ws = plan.encode_only(dev(A), dev(B))
+    q0, s0 = plan.quantized_operand(ws, 256, 256, 256, 4, "A")
+    r0, t0 = plan.quantized_operand(ws, 256, 256, 256, 4, "B")
+    ws = plan.encode_only(dev(A * np.float32(2.0 ** 9)), dev(B * np.float32(2.0 ** -13)))
+    q1, s1 = plan.quantized_operand(ws, 256, 256, 256, 4, "A")
+    r1, t1 = plan.quantized_operand(ws, 256, 256, 256, 4, "B")
+    assert np.array_equal(q0, q1) and np.array_equal(r0, r1)
+    assert np.array_equal(s1, s0 * np.float32(2.0 ** 9)) and np.array_equal(t1, t0 * np.float32(2.0 ** -13))
+
+
+def test_term_permutation_and_cubic_realization_properties():
+    # permuting the terms of a realization only changes the summation order of the decode;
+    # the rank-8 cubic realization at one level quantizes the same blocks as the cubic product
+    A, B = Wl.gaussian(512, 512, 512, 8)
+    a, b = dev(A), dev(B)
+    U, V, W = P.get("winograd")
+    perm = np.array([3, 0, 6, 1, 5, 2, 4])
+    c0 = fmm.Plan(U, V, W, levels=1, scale_mode="ue8m0").matmul(a, b).cpu().numpy().astype(np.float64)
+    c1 = fmm.Plan(U[perm], V[perm], W[perm], levels=1, scale_mode="ue8m0").matmul(a, b).cpu().numpy().astype(np.float64)
+    assert np.linalg.norm(c0 - c1) / np.linalg.norm(c0) < 1e-6
+    c8 = fmm.Plan(*P.get("cubic8"), levels=1, scale_mode="fp32").matmul(a, b).cpu().numpy().astype(np.float64)
+    cc = fmm.Plan(levels=0, scale_mode="fp32").matmul(a, b).cpu().numpy().astype(np.float64)
+    assert np.linalg.norm(c8 - cc) / np.linalg.norm(cc) < 1e-6
+
+
+def test_rademacher_operands_strassen_is_exact_up_to_scale_rounding():
+    # Sec. 4.3: on +-1 operands Strassen's combinations are exactly representable after block scaling
+    A, B = Wl.rademacher(256, 256, 256, 0)
+    a, b = dev(A), dev(B)
+    ref = fmm.fmm_ref_gemm_fp64(a, b)
+    es = fmm.rel_frobenius(make_plan("strassen", 1, 32, "fp32").matmul(a, b), ref)
+    ep = fmm.rel_frobenius(make_plan("phi_optimal", 1, 32, "fp32").matmul(a, b), ref)
+    assert es < 1e-6 and ep > 1e-3
+    es_mx = fmm.rel_frobenius(make_plan("strassen", 1, 32, "ue8m0").matmul(a, b), ref)
+    assert es_mx == 0.0          # power-of-two scales: exact
+
+
+def test_bounded_wait_runs_out_and_leaves_the_context_usable():
+    plan = make_plan("strassen", 1, 32, "ue8m0")
+    assert plan.device_status() == (0, 0)
+    plan.selftest_bounded_wait(2_000_000)                 # 2 ms limit on a barrier nothing signals
+    torch.cuda.synchronize()
+    st, code = plan.device_status()
+    assert st == 8 and code == 901                        # FMM_ERR_DEVICE_TIMEOUT, self-test location
+    plan.device_status_clear()
+    assert plan.device_status() == (0, 0)
+    # the context still works: a real product after the timed-out wait matches the oracle
+    A, B = Wl.gaussian(256, 256, 256, 2)
+    got = plan.matmul(dev(A), dev(B)).cpu().numpy().astype(np.float64)
+    want = O.fused_fmm(A, B, *P.get("strassen"), levels=1, blk=32, mode=O.SCALE_UE8M0)
+    assert np.linalg.norm(got - want) / np.linalg.norm(want) < 1e-5
+    assert plan.device_status() == (0, 0)
