@@ -32,6 +32,9 @@ CONFIGS = {
     "c2": dict(shape=(4096, 4096, 4096), families=["gaussian", "uniform"], trials=50, names=ALL, levels=[1]),
     "c3": dict(shape=(8192, 8192, 8192), families=["gaussian"], trials=3, names=["cubic", "strassen", "phi_optimal"], levels=[1, 2]),
     "c4": dict(shape=(16384, 8192, 8192), families=["llm"], trials=3, names=ALL, levels=[1]),
+    # operand-family controls (Sec. 4.3 / Table E.8): unit-variance families and Rademacher +-1 / +-10 cells
+    "c6": dict(shape=(2048, 2048, 2048), families=["gaussian", "unit_uniform", "unit_laplace", "unit_t5", "rademacher", "rademacher10"],
+               trials=8, names=ALL, levels=[1]),
     "c5": dict(shape=(2048, 2048, 2048), families=["scaled_gaussian", "student_t3"], trials=256, names=ALL, levels=[1, 2, 3]),
 }
 
@@ -104,8 +107,9 @@ def summarise(path, file=sys.stdout):
             e = np.array([seeds[s]["rel_frobenius"] for s in sorted(seeds)])
             pooled = math.sqrt(sum(seeds[s]["sum_sq_diff"] for s in seeds) / sum(seeds[s]["sum_sq_ref"] for s in seeds))
             common = [s for s in seeds if s in cubic]
-            ratio = (np.mean([seeds[s]["rel_frobenius"] for s in common]) /
-                     np.mean([cubic[s]["rel_frobenius"] for s in common])) if common else float("nan")
+            cub = np.mean([cubic[s]["rel_frobenius"] for s in common]) if common else 0.0
+            # operands the cubic product represents (almost) exactly make the ratio meaningless
+            ratio = np.mean([seeds[s]["rel_frobenius"] for s in common]) / cub if cub > 1e-6 else float("nan")
             pred = PREDICTED.get(name, float("nan")) ** max(lv, 1) if name != "cubic" else 1.0
             rows.append((g, name, lv, len(e), e.mean(), e.std(), pooled, ratio, pred))
     print("| config | family | scales | blk | realization | levels | trials | mean rel. error | sd | pooled RMS | ratio vs cubic | sqrt(Phi/8)^l |", file=file)

@@ -72,6 +72,32 @@ def small_integers(M, K, N, seed, amp=8):
     return A, B
 
 
+def unit_uniform(M, K, N, seed):
+    """iid U(-sqrt 3, sqrt 3): unit variance."""
+    A, B = uniform(M, K, N, seed)
+    r3 = np.float32(np.sqrt(3.0))
+    return A * r3, B * r3
+
+
+def unit_laplace(M, K, N, seed):
+    """iid Laplace with unit variance (scale 1/sqrt 2)."""
+    A = _rng(seed, 0).laplace(0.0, 1.0 / np.sqrt(2.0), (M, K)).astype(np.float32)
+    B = _rng(seed, 1).laplace(0.0, 1.0 / np.sqrt(2.0), (K, N)).astype(np.float32)
+    return A, B
+
+
+def unit_t5(M, K, N, seed):
+    """iid Student-t(nu = 5) scaled to unit variance (variance of t5 is 5/3)."""
+    c = np.sqrt(3.0 / 5.0)
+    A = (_rng(seed, 0).standard_t(5.0, (M, K)) * c).astype(np.float32)
+    B = (_rng(seed, 1).standard_t(5.0, (K, N)) * c).astype(np.float32)
+    return A, B
+
+
+def rademacher10(M, K, N, seed):
+    return rademacher(M, K, N, seed, scale=10.0)
+
+
 FAMILIES = {
     "gaussian": gaussian,
     "uniform": uniform,
@@ -80,4 +106,8 @@ FAMILIES = {
     "student_t3": student_t3,
     "rademacher": rademacher,
     "small_integers": small_integers,
+    "unit_uniform": unit_uniform,
+    "unit_laplace": unit_laplace,
+    "unit_t5": unit_t5,
+    "rademacher10": rademacher10,
 }
