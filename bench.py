@@ -252,17 +252,19 @@ def run_ours(args):
                    "multiply_tflops": flops_alg / (mul_ms * 1e-3) / 1e12},
         "device_status": status[1],
     }
-    # dominant kernel = the tcgen05 product kernel.  DRAM traffic per launch: dram__bytes_read + write from the
-    # ncu capture at n = 4096 (profiles/fmm_gemm_kernel_n4096.md), scaled by the units processed (bytes ~ M*N)
-    measured_4096 = {("fp32", 32): 136.4e6, ("ue8m0", 32): 151.0e6}.get((args.scale_mode, args.block_k))
+    # dominant kernel = the tcgen05 product kernel.  DRAM traffic per launch: dram__bytes_read + write from one-pass
+    # ncu captures of this command (profiles/fmm_gemm_kernel_dram_traffic.md).  At n = 8192 the live C tiles and the
+    # operand streams no longer fit L2 together, so traffic does not scale with M*N: only measured sizes are reported.
+    measured = {("fp32", 32, 8192): 1542.4e6, ("ue8m0", 32, 8192): 1662.8e6,
+                ("fp32", 32, 4096): 136.4e6, ("ue8m0", 32, 4096): 151.0e6}
     traffic = None
-    if measured_4096 is not None and args.levels == 1:
-        traffic = measured_4096 * (M * N) / (4096.0 * 4096.0)
+    if args.levels == 1 and M == N == K and args.realization == "phi_optimal":
+        traffic = measured.get((args.scale_mode, args.block_k, M))
     t_roof_ms = (flops_alg / (fp8_peak * 1e12) + (enc_bytes + gemm_bytes) / (hbm * 1e9)) * 1e3
     out["roofline"] = {"kernel": "fmm_gemm_kernel", "bound": "tensor",
                        "achieved": flops_alg / (mul_ms * 1e-3) / 1e12, "peak": fp8_peak, "unit": "TFLOP/s",
                        "frac": flops_alg / (mul_ms * 1e-3) / 1e12 / fp8_peak, "traffic": traffic,
-                       "traffic_unit": "bytes per launch (ncu at n=4096, scaled)", "algorithmic_bytes": gemm_bytes,
+                       "traffic_unit": "bytes per launch (ncu dram__bytes_read.sum + dram__bytes_write.sum at this size)", "algorithmic_bytes": gemm_bytes,
                        "peak_source": f"2 x {pk['source']} bf16 burst ({pk['bf16_tflops']} TF/s)",
                        "combined_roofline_ms": t_roof_ms, "combined_frac": t_roof_ms / ms_step}
     if args.scale_mode == "fp32":

@@ -39,7 +39,6 @@ constexpr int NUM_THREADS = (EPI_WARP0 + EPI_WARPS) * 32;
 constexpr int REGS_AT_LAUNCH = 168, REGS_CTRL = 56, REGS_EPI = 224;
 static_assert(EPI_WARP0 * 32 * REGS_CTRL + EPI_WARPS * 32 * REGS_EPI <= NUM_THREADS * REGS_AT_LAUNCH, "register pool");
 static_assert(NUM_THREADS * (REGS_AT_LAUNCH + 8) > 65536, "REGS_AT_LAUNCH must be the launch-bound maximum");
-constexpr int STAGING_BYTES = 32 * 128; // 32 rows x 32 fp32 per epilogue warp and buffer
 
 template <int BN, int MODE, int BLK, int NCTA>
 struct Cfg {
@@ -47,16 +46,21 @@ struct Cfg {
     static constexpr int BROWS = BN / NCTA;                  // T_r rows this CTA loads per stage
     static constexpr int A_BYTES = BM * BK;
     static constexpr int B_BYTES = BROWS * BK;
-    // The UE8M0 pair kernel is bound by operand-load latency under L2 contention: it trades one
-    // epilogue staging buffer per warp for a fifth pipeline stage.
+    // The UE8M0 pair kernel is bound by operand-load latency under L2 contention: it trades epilogue
+    // staging space for more pipeline stages.
     static constexpr int STAGING_BUFS = (MX && NCTA == 2) ? 1 : 2;
-    static constexpr int STAGES = (MX && NCTA == 2) ? 5 : ((A_BYTES + B_BYTES) > 40000 ? 3 : 4);
+    static constexpr int STAGES = (MX && NCTA == 2) ? 6 : ((A_BYTES + B_BYTES) > 40000 ? 3 : 4);
+    // output chunk of one epilogue warp: 32 rows x CH fp32, staged in shared memory for one TMA store
+    // (the UE8M0 pair kernel halves it: with one narrow buffer per warp a sixth operand stage fits)
+    static constexpr int CH = (MX && NCTA == 2) ? 16 : 32;
+    static constexpr int STAGING_BYTES = 32 * CH * 4;
     static constexpr int SFB_ATOMS = BN / 128;
     static constexpr int SF_STAGE_BYTES = MX ? (512 + SFB_ATOMS * 512) : 0;
     static constexpr int KB_PER_STAGE = BK / BLK;
     static constexpr int SB_STAGES = STAGES + 1;
     static constexpr int SB_STAGE_BYTES = MX ? 0 : KB_PER_STAGE * BN * 4;
     static constexpr int TX_BYTES = NCTA * (A_BYTES + B_BYTES + SF_STAGE_BYTES);
+    static constexpr int TX_BYTES_HALF = NCTA * (A_BYTES + B_BYTES / 2 + 1024);   // half-width item: one SFB atom
     static constexpr int OFF_A = 0;
     static constexpr int OFF_B = OFF_A + STAGES * A_BYTES;
     static constexpr int OFF_STG = OFF_B + STAGES * B_BYTES;
@@ -73,9 +77,37 @@ struct Cfg {
     static constexpr int ACC_BUFS = MX ? 1 : (512 / BN) / GPB;        // ring of (GPB x BN)-column super-buffers
     static constexpr int SF_COLS = 4 + 4 * SFB_ATOMS;
     static constexpr int CW = BN / 2;      // columns per epilogue warp
+    // Tail split (UE8M0, 256-column tiles): when the last wave of tile positions would occupy at most half
+    // of the CTAs (pairs), each of those positions is cut into two 128-column items, so the last wave
+    // takes about half as long.  Every item still runs all its terms in one CTA (pair): no output tile is
+    // shared between CTAs and the summation order stays fixed.
+    static constexpr bool SPLIT = MX && BN == 256;
     static_assert(SMEM_BYTES <= 232448, "shared memory budget");
     static_assert(!MX || BN + STAGES * SF_COLS <= 512, "TMEM budget");
 };
+
+#ifndef FMM_HINT_OPERANDS
+#define FMM_HINT_OPERANDS 0     // L2 policy of the operand tile loads: 0 default, 1 evict-first, 2 evict-last
+#endif
+#ifndef FMM_HINT_C
+// L2 policy of the output stores / add-reductions.  Each C tile is updated once per term that feeds it; between
+// two updates a whole term's operands stream through L2, so the tiles are marked evict-last (measured at
+// n = 8192: fewer write-backs of half-accumulated tiles, product kernel 3 % faster; an evict-first policy on
+// the operand loads was slower).
+#define FMM_HINT_C 2
+#endif
+#if FMM_HINT_OPERANDS
+#define LOAD_OP(dst, tm, x, y, bar) tma_load_2d_hint<NCTA>(dst, tm, x, y, bar, pol_op)
+#else
+#define LOAD_OP(dst, tm, x, y, bar) tma_load_2d<NCTA>(dst, tm, x, y, bar)
+#endif
+#if FMM_HINT_C
+#define STORE_C(tm, x, y, src) tma_store_2d_hint(tm, x, y, src, pol_c)
+#define REDUCE_C(tm, x, y, src) tma_reduce_add_2d_hint(tm, x, y, src, pol_c)
+#else
+#define STORE_C(tm, x, y, src) tma_store_2d(tm, x, y, src)
+#define REDUCE_C(tm, x, y, src) tma_reduce_add_2d(tm, x, y, src)
+#endif
 
 #ifdef FMM_TIMING
 #define TCLK() clock64()
@@ -140,6 +172,7 @@ struct KParams {
     const uint8_t* sa; const uint8_t* sb;   // scale arrays (bytes); fp32 mode only
     long long sa_term, sb_term;
     int m, n, k, terms;
+    int split_from, items;                  // positions >= split_from are cut into two 128-column items
     const int* out_start; const FmmOutEntry* out;
     int* status;
 };
@@ -148,7 +181,8 @@ template <int BN, int MODE, int BLK, int NCTA>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                 const __grid_constant__ CUtensorMap tmC, const __grid_constant__ CUtensorMap tmSFA,
-                const __grid_constant__ CUtensorMap tmSFB, const KParams p)
+                const __grid_constant__ CUtensorMap tmSFB, const __grid_constant__ CUtensorMap tmBh,
+                const __grid_constant__ CUtensorMap tmSFBh, const KParams p)
 {
     using C = Cfg<BN, MODE, BLK, NCTA>;
     extern __shared__ uint8_t smem_raw[];
@@ -195,7 +229,10 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     const uint32_t tmem_base = *tmem_slot;
 
     const int tiles_n = p.n / BN;
-    const int positions = (p.m / (BM * NCTA)) * tiles_n;
+    // work item w -> tile position, column offset inside the position, half-width flag
+    auto item_pos = [&](int w) { return (C::SPLIT && w >= p.split_from) ? p.split_from + ((w - p.split_from) >> 1) : w; };
+    auto item_half = [&](int w) { return C::SPLIT && w >= p.split_from; };
+    auto item_coff = [&](int w) { return (C::SPLIT && w >= p.split_from) ? ((w - p.split_from) & 1) * (BN / 2) : 0; };
     const int kstages = p.k / BK;
     const int nkb = p.k / BLK;
     const int row_blocks_a = p.m / 128, row_blocks_b = p.n / 128;
@@ -208,7 +245,14 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             int stage = 0; uint32_t phase = 0;
             int ss = 0; uint32_t sphase = 0;
             bool ok = true;
-            for (int pos = unit; pos < positions && ok; pos += units) {
+#if FMM_HINT_OPERANDS == 1
+            const uint64_t pol_op = policy_evict_first();
+#elif FMM_HINT_OPERANDS == 2
+            const uint64_t pol_op = policy_evict_last();
+#endif
+            for (int w = unit; w < p.items && ok; w += units) {
+                const int pos = item_pos(w), coff = item_coff(w);
+                const bool half = item_half(w);
                 const int tm = pos / tiles_n, tn = pos % tiles_n;
                 const int row_blk = tm * NCTA + cta_rank;                 // 128-row block of S_r this CTA owns
                 for (int t = 0; t < p.terms && ok; ++t) {
@@ -223,15 +267,29 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                         if (++stage == C::STAGES) { stage = 0; phase ^= 1u; }
                         continue;
 #endif
-                        if (leader) mbar_expect_tx(bar_full(stage), C::TX_BYTES);
-                        tma_load_2d<NCTA>(base + C::OFF_A + stage * C::A_BYTES, &tmA, ks * BK, t * p.m + row_blk * BM, fb);
-                        tma_load_2d<NCTA>(base + C::OFF_B + stage * C::B_BYTES, &tmB, ks * BK,
-                                          t * p.n + tn * BN + cta_rank * C::BROWS, fb);
+#if defined(FMM_EXP_SKIP_A)
+                        // timing experiment only: A tiles not loaded on (some) stages
+                        const bool load_a = (ks % FMM_EXP_SKIP_A) == 0 && FMM_EXP_SKIP_A < 100;
+                        if (leader) mbar_expect_tx(bar_full(stage), (half ? C::TX_BYTES_HALF : C::TX_BYTES) - (load_a ? 0 : NCTA * C::A_BYTES));
+                        if (load_a)
+#else
+                        if (leader) mbar_expect_tx(bar_full(stage), half ? C::TX_BYTES_HALF : C::TX_BYTES);
+#endif
+                        LOAD_OP(base + C::OFF_A + stage * C::A_BYTES, &tmA, ks * BK, t * p.m + row_blk * BM, fb);
+                        if (!half)
+                            LOAD_OP(base + C::OFF_B + stage * C::B_BYTES, &tmB, ks * BK,
+                                    t * p.n + tn * BN + cta_rank * C::BROWS, fb);
+                        else
+                            LOAD_OP(base + C::OFF_B + stage * C::B_BYTES, &tmBh, ks * BK,
+                                    t * p.n + tn * BN + coff + cta_rank * (C::BROWS / 2), fb);
                         if (C::MX) {
                             // scale tiles: 512-byte atoms, ordered [term][k quad][128-row block]
                             const uint32_t sf = base + C::OFF_SF + stage * C::SF_STAGE_BYTES;
                             tma_load_2d<NCTA>(sf, &tmSFA, 0, (t * (nkb >> 2) + ks) * row_blocks_a + row_blk, fb);
-                            tma_load_2d<NCTA>(sf + 512, &tmSFB, 0, (t * (nkb >> 2) + ks) * row_blocks_b + tn * C::SFB_ATOMS, fb);
+                            if (!half)
+                                tma_load_2d<NCTA>(sf + 512, &tmSFB, 0, (t * (nkb >> 2) + ks) * row_blocks_b + tn * C::SFB_ATOMS, fb);
+                            else
+                                tma_load_2d<NCTA>(sf + 512, &tmSFBh, 0, (t * (nkb >> 2) + ks) * row_blocks_b + tn * C::SFB_ATOMS + coff / 128, fb);
                         } else {
                             if (!mbar_wait(bar_sempty(ss), sphase ^ 1u, ctl, 102)) { ok = false; break; }
                             mbar_expect_tx(bar_sfull(ss), C::SB_STAGE_BYTES);
@@ -255,10 +313,13 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             int buf = 0; uint32_t bphase = 0;
             bool ok = true;
             constexpr uint32_t MDIM = (uint32_t)(BM * NCTA) >> 4;
-            uint32_t idesc;
-            if (C::MX) idesc = (1u << 23) | ((uint32_t)(BN >> 3) << 17) | (MDIM << 24);
-            else idesc = (1u << 4) | ((uint32_t)(BN >> 3) << 17) | (MDIM << 24);
-            for (int pos = unit; pos < positions && ok; pos += units) {
+            uint32_t idesc_full;
+            if (C::MX) idesc_full = (1u << 23) | ((uint32_t)(BN >> 3) << 17) | (MDIM << 24);
+            else idesc_full = (1u << 4) | ((uint32_t)(BN >> 3) << 17) | (MDIM << 24);
+            for (int w = unit; w < p.items && ok; w += units) {
+                const bool half = item_half(w);
+                // a half-width item is the same instruction with N = BN/2
+                const uint32_t idesc = half ? (idesc_full & ~(0x3Fu << 17)) | ((uint32_t)(BN >> 4) << 17) : idesc_full;
                 for (int t = 0; t < p.terms && ok; ++t) {
                     if (C::MX) {
                         const long long tw = TCLK();
@@ -281,7 +342,7 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                             tc_cp_32x128b_warpx4<NCTA>(tsfa, make_sf_desc(sf));
 #pragma unroll
                             for (int h = 0; h < C::SFB_ATOMS; ++h)
-                                tc_cp_32x128b_warpx4<NCTA>(tsfb + 4 * h, make_sf_desc(sf + 512 + h * 512));
+                                if (h == 0 || !half) tc_cp_32x128b_warpx4<NCTA>(tsfb + 4 * h, make_sf_desc(sf + 512 + h * 512));
 #endif
 #pragma unroll
                             for (int j = 0; j < BK / 32; ++j) {
@@ -322,9 +383,8 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         const int e = warp - EPI_WARP0;
         const int q = warp & 3;            // TMEM lane quadrant this warp may access
         const int h = e >> 2;              // column half
-        const uint32_t stg = base + C::OFF_STG + e * C::STAGING_BUFS * STAGING_BYTES;
-        uint8_t* stg_ptr = base_ptr + C::OFF_STG + e * C::STAGING_BUFS * STAGING_BYTES;
-        const uint32_t lane_taddr = tmem_base + ((uint32_t)(q * 32) << 16) + h * C::CW;
+        const uint32_t stg = base + C::OFF_STG + e * C::STAGING_BUFS * C::STAGING_BYTES;
+        uint8_t* stg_ptr = base_ptr + C::OFF_STG + e * C::STAGING_BUFS * C::STAGING_BYTES;
         // the accumulator-free signal goes to the MMA issuer, which lives in the even CTA
         auto release_acc = [&](int b) {
             if (NCTA == 2) mbar_arrive_cluster(bar_tempty(b) & PEER_BIT_MASK); else mbar_arrive(bar_tempty(b));
@@ -333,11 +393,21 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         int ss = 0; uint32_t sphase = 0;
         uint32_t store_cnt = 0;
         bool ok = true;
+#if FMM_HINT_C == 1
+        const uint64_t pol_c = policy_evict_first();
+#elif FMM_HINT_C == 2
+        const uint64_t pol_c = policy_evict_last();
+#endif
         uint32_t accu[C::MX ? C::CW : 1];               // UE8M0: raw fp32 bits drained from TMEM
         unsigned long long acc2[C::MX ? 1 : C::CW / 2]; // FP32: promoted accumulators, two columns per register pair
-        for (int pos = unit; pos < positions && ok; pos += units) {
+        for (int w = unit; w < p.items && ok; w += units) {
+            const int pos = item_pos(w), coff = item_coff(w);
             const int tm = pos / tiles_n, tn = pos % tiles_n;
             const int row_in_leaf = (tm * NCTA + cta_rank) * BM + q * 32;
+            // columns this warp owns: half of the item's width, in 32-column chunks
+            const int cw = item_half(w) ? C::CW / 2 : C::CW;
+            const int nch = cw / 32;
+            const uint32_t lane_taddr = tmem_base + ((uint32_t)(q * 32) << 16) + h * cw;
             for (int t = 0; t < p.terms && ok; ++t) {
                 if (C::MX) {
                     const long long tw = TCLK();
@@ -345,7 +415,8 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                     TADD(3, tw);
                     tc_fence_after();
 #pragma unroll
-                    for (int c = 0; c < C::CW / 32; ++c) tmem_ld32(lane_taddr + c * 32, &accu[c * 32]);
+                    for (int c = 0; c < C::CW / 32; ++c)
+                        if (c < nch) tmem_ld32(lane_taddr + c * 32, &accu[c * 32]);
                     tmem_ld_wait();
                     tc_fence_before();
                     __syncwarp();
@@ -425,31 +496,39 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                 for (int o = o0; o < o1; ++o) {
                     const FmmOutEntry ent = p.out[o];
                     const int row0 = ent.row_off * p.m + row_in_leaf;
-                    const int col0 = ent.col_off * p.n + tn * BN + h * C::CW;
+                    const int col0 = ent.col_off * p.n + tn * BN + coff + h * cw;
 #pragma unroll
-                    for (int c = 0; c < C::CW / 32; ++c) {
+                    for (int c = 0; c < C::CW / C::CH; ++c) {
+                        if (c * C::CH >= cw) break;
                         const uint32_t b = store_cnt & (C::STAGING_BUFS - 1);
                         if (lane == 0) bulk_wait_read<C::STAGING_BUFS - 1>();   // the buffer about to be rewritten has been read
                         __syncwarp();
-                        uint8_t* dst = stg_ptr + b * STAGING_BYTES + lane * 128;
+                        // one row of the chunk per lane; 16-byte pieces permuted as the tensor map's swizzle expects
+                        uint8_t* dst = stg_ptr + b * C::STAGING_BYTES + lane * (C::CH * 4);
+                        const int swz = (C::CH == 32) ? (lane & 7) : ((lane >> 1) & 3);
 #pragma unroll
-                        for (int i4 = 0; i4 < 8; ++i4) {
+                        for (int i4 = 0; i4 < C::CH / 4; ++i4) {
                             float4 v;
                             if (C::MX) {
-                                v.x = __uint_as_float(accu[c * 32 + i4 * 4 + 0]); v.y = __uint_as_float(accu[c * 32 + i4 * 4 + 1]);
-                                v.z = __uint_as_float(accu[c * 32 + i4 * 4 + 2]); v.w = __uint_as_float(accu[c * 32 + i4 * 4 + 3]);
+                                v.x = __uint_as_float(accu[c * C::CH + i4 * 4 + 0]); v.y = __uint_as_float(accu[c * C::CH + i4 * 4 + 1]);
+                                v.z = __uint_as_float(accu[c * C::CH + i4 * 4 + 2]); v.w = __uint_as_float(accu[c * C::CH + i4 * 4 + 3]);
                             } else {
-                                unpack2(acc2[c * 16 + i4 * 2], v.x, v.y);
-                                unpack2(acc2[c * 16 + i4 * 2 + 1], v.z, v.w);
+                                unpack2(acc2[c * (C::CH / 2) + i4 * 2], v.x, v.y);
+                                unpack2(acc2[c * (C::CH / 2) + i4 * 2 + 1], v.z, v.w);
                             }
                             v.x *= ent.w; v.y *= ent.w; v.z *= ent.w; v.w *= ent.w;
-                            *reinterpret_cast<float4*>(dst + ((i4 ^ (lane & 7)) << 4)) = v;
+                            *reinterpret_cast<float4*>(dst + ((i4 ^ swz) << 4)) = v;
                         }
                         fence_proxy_async();
                         __syncwarp();
                         if (lane == 0) {
-                            if (ent.first) tma_store_2d(&tmC, col0 + c * 32, row0, stg + b * STAGING_BYTES);
-                            else tma_reduce_add_2d(&tmC, col0 + c * 32, row0, stg + b * STAGING_BYTES);
+#if defined(FMM_EXP_NO_OUT)
+#elif defined(FMM_EXP_STORE_ONLY)
+                            STORE_C(&tmC, col0 + c * C::CH, row0, stg + b * C::STAGING_BYTES);
+#else
+                            if (ent.first) STORE_C(&tmC, col0 + c * C::CH, row0, stg + b * C::STAGING_BYTES);
+                            else REDUCE_C(&tmC, col0 + c * C::CH, row0, stg + b * C::STAGING_BYTES);
+#endif
                             bulk_commit();
                         }
                         ++store_cnt;
@@ -520,11 +599,12 @@ template <int BN, int MODE, int BLK, int NCTA>
 fmm_status_t launch(const GemmParams& g, cudaStream_t st)
 {
     using C = Cfg<BN, MODE, BLK, NCTA>;
-    CUtensorMap tmA, tmB, tmC, tmSFA, tmSFB;
+    CUtensorMap tmA, tmB, tmC, tmSFA, tmSFB, tmBh, tmSFBh;
     const CUtensorMapSwizzle SW = CU_TENSOR_MAP_SWIZZLE_128B;
     if (!make_map_2d(&tmA, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, g.qa, (uint64_t)g.k, (uint64_t)g.terms * g.m, BK, BM, SW)) return FMM_ERR_CUDA;
     if (!make_map_2d(&tmB, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, g.qb, (uint64_t)g.k, (uint64_t)g.terms * g.n, BK, C::BROWS, SW)) return FMM_ERR_CUDA;
-    if (!make_map_2d(&tmC, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, g.C, (uint64_t)g.Nfull, (uint64_t)g.Mfull, 32, 32, SW)) return FMM_ERR_CUDA;
+    if (!make_map_2d(&tmC, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, g.C, (uint64_t)g.Nfull, (uint64_t)g.Mfull, C::CH, 32,
+                     C::CH == 32 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B)) return FMM_ERR_CUDA;
     if (C::MX) {
         // scale tiles as rows of 128 uint32 (one 512-byte atom per row)
         const uint64_t atoms_a = (uint64_t)g.terms * (g.k / 128) * (g.m / 128), atoms_b = (uint64_t)g.terms * (g.k / 128) * (g.n / 128);
@@ -532,6 +612,13 @@ fmm_status_t launch(const GemmParams& g, cudaStream_t st)
         if (!make_map_2d(&tmSFB, CU_TENSOR_MAP_DATA_TYPE_UINT32, 4, g.sb, 128, atoms_b, 128, C::SFB_ATOMS, CU_TENSOR_MAP_SWIZZLE_NONE)) return FMM_ERR_CUDA;
     } else {
         tmSFA = tmA; tmSFB = tmB;       // unused in this mode
+    }
+    tmBh = tmB; tmSFBh = tmSFB;
+    if (C::SPLIT) {
+        // half-width items: half as many rows of T_r per CTA, one scale atom
+        const uint64_t atoms_b = (uint64_t)g.terms * (g.k / 128) * (g.n / 128);
+        if (!make_map_2d(&tmBh, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, g.qb, (uint64_t)g.k, (uint64_t)g.terms * g.n, BK, C::BROWS / 2, SW)) return FMM_ERR_CUDA;
+        if (!make_map_2d(&tmSFBh, CU_TENSOR_MAP_DATA_TYPE_UINT32, 4, g.sb, 128, atoms_b, 128, 1, CU_TENSOR_MAP_SWIZZLE_NONE)) return FMM_ERR_CUDA;
     }
     static bool attr_set = false;
     if (!attr_set) {
@@ -547,10 +634,14 @@ fmm_status_t launch(const GemmParams& g, cudaStream_t st)
     const int positions = (g.m / (BM * NCTA)) * (g.n / BN);
     const int max_units = sms / NCTA;
     const int units = positions < max_units ? positions : max_units;
+    const int tail = positions % units;
+    const bool split = C::SPLIT && tail > 0 && 2 * tail <= units;
     KParams kp;
     kp.sa = static_cast<const uint8_t*>(g.sa); kp.sb = static_cast<const uint8_t*>(g.sb);
     kp.sa_term = g.sa_term; kp.sb_term = g.sb_term;
     kp.m = g.m; kp.n = g.n; kp.k = g.k; kp.terms = g.terms;
+    kp.split_from = split ? positions - tail : positions;
+    kp.items = positions + (split ? tail : 0);
     kp.out_start = g.out_start; kp.out = g.out; kp.status = g.status;
 
     cudaLaunchConfig_t cfg;
@@ -563,7 +654,7 @@ fmm_status_t launch(const GemmParams& g, cudaStream_t st)
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = NCTA; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
-    cudaError_t ce = cudaLaunchKernelEx(&cfg, fmm_gemm_kernel<BN, MODE, BLK, NCTA>, tmA, tmB, tmC, tmSFA, tmSFB, kp);
+    cudaError_t ce = cudaLaunchKernelEx(&cfg, fmm_gemm_kernel<BN, MODE, BLK, NCTA>, tmA, tmB, tmC, tmSFA, tmSFB, tmBh, tmSFBh, kp);
     if (ce != cudaSuccess) { cudaGetLastError(); return FMM_ERR_CUDA; }
     return FMM_OK;
 }

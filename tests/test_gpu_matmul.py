@@ -30,6 +30,10 @@ CASES = [
     ("phi_optimal", 1, (1024, 1024, 1024), 32, "ue8m0", "gaussian"),
     ("phi_optimal", 1, (1024, 1024, 1024), 32, "fp32", "gaussian"),
     ("phi_optimal", 1, (1024, 1024, 1024), 128, "fp32", "gaussian"),
+    # more tile positions than CTA pairs / CTAs on a 148-SM part, with a short last wave: the product
+    # kernel cuts the last positions into half-width items (80 positions on 74 pairs; 152 on 148 CTAs)
+    ("strassen", 1, (5120, 512, 4096), 32, "ue8m0", "gaussian"),
+    ("phi_optimal", 1, (4864, 256, 4096), 32, "ue8m0", "uniform"),
 ]
 
 
