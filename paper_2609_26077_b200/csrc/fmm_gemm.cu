@@ -86,29 +86,6 @@ struct Cfg {
     static_assert(!MX || BN + STAGES * SF_COLS <= 512, "TMEM budget");
 };
 
-#ifndef FMM_HINT_OPERANDS
-#define FMM_HINT_OPERANDS 0     // L2 policy of the operand tile loads: 0 default, 1 evict-first, 2 evict-last
-#endif
-#ifndef FMM_HINT_C
-// L2 policy of the output stores / add-reductions.  Each C tile is updated once per term that feeds it; between
-// two updates a whole term's operands stream through L2, so the tiles are marked evict-last (measured at
-// n = 8192: fewer write-backs of half-accumulated tiles, product kernel 3 % faster; an evict-first policy on
-// the operand loads was slower).
-#define FMM_HINT_C 2
-#endif
-#if FMM_HINT_OPERANDS
-#define LOAD_OP(dst, tm, x, y, bar) tma_load_2d_hint<NCTA>(dst, tm, x, y, bar, pol_op)
-#else
-#define LOAD_OP(dst, tm, x, y, bar) tma_load_2d<NCTA>(dst, tm, x, y, bar)
-#endif
-#if FMM_HINT_C
-#define STORE_C(tm, x, y, src) tma_store_2d_hint(tm, x, y, src, pol_c)
-#define REDUCE_C(tm, x, y, src) tma_reduce_add_2d_hint(tm, x, y, src, pol_c)
-#else
-#define STORE_C(tm, x, y, src) tma_store_2d(tm, x, y, src)
-#define REDUCE_C(tm, x, y, src) tma_reduce_add_2d(tm, x, y, src)
-#endif
-
 #ifdef FMM_TIMING
 #define TCLK() clock64()
 #define TADD(slot, t0) do { if (blockIdx.x == 0 && lane == 0) tim[slot] += clock64() - (t0); } while (0)
@@ -130,11 +107,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const C
 {
     uint32_t spins = 0;
     uint64_t t0 = 0;
-#ifdef FMM_EXP_TEST_WAIT
-    while (!mbar_test_wait(bar, parity)) {
-#else
     while (!mbar_try_wait(bar, parity)) {
-#endif
         if ((++spins & 0x3FFu) == 0) {
             if (*ctl.abort_flag) return false;
             const uint64_t now = global_timer();
@@ -245,11 +218,6 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             int stage = 0; uint32_t phase = 0;
             int ss = 0; uint32_t sphase = 0;
             bool ok = true;
-#if FMM_HINT_OPERANDS == 1
-            const uint64_t pol_op = policy_evict_first();
-#elif FMM_HINT_OPERANDS == 2
-            const uint64_t pol_op = policy_evict_last();
-#endif
             for (int w = unit; w < p.items && ok; w += units) {
                 const int pos = item_pos(w), coff = item_coff(w);
                 const bool half = item_half(w);
@@ -262,26 +230,14 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                         TADD(0, tw);
                         // completion is counted on the even CTA's barrier; only that CTA arms it
                         const uint32_t fb = (NCTA == 2) ? (bar_full(stage) & PEER_BIT_MASK) : bar_full(stage);
-#ifdef FMM_EXP_NO_TMA
-                        if (leader) mbar_arrive(bar_full(stage));
-                        if (++stage == C::STAGES) { stage = 0; phase ^= 1u; }
-                        continue;
-#endif
-#if defined(FMM_EXP_SKIP_A)
-                        // timing experiment only: A tiles not loaded on (some) stages
-                        const bool load_a = (ks % FMM_EXP_SKIP_A) == 0 && FMM_EXP_SKIP_A < 100;
-                        if (leader) mbar_expect_tx(bar_full(stage), (half ? C::TX_BYTES_HALF : C::TX_BYTES) - (load_a ? 0 : NCTA * C::A_BYTES));
-                        if (load_a)
-#else
                         if (leader) mbar_expect_tx(bar_full(stage), half ? C::TX_BYTES_HALF : C::TX_BYTES);
-#endif
-                        LOAD_OP(base + C::OFF_A + stage * C::A_BYTES, &tmA, ks * BK, t * p.m + row_blk * BM, fb);
+                        tma_load_2d<NCTA>(base + C::OFF_A + stage * C::A_BYTES, &tmA, ks * BK, t * p.m + row_blk * BM, fb);
                         if (!half)
-                            LOAD_OP(base + C::OFF_B + stage * C::B_BYTES, &tmB, ks * BK,
-                                    t * p.n + tn * BN + cta_rank * C::BROWS, fb);
+                            tma_load_2d<NCTA>(base + C::OFF_B + stage * C::B_BYTES, &tmB, ks * BK,
+                                              t * p.n + tn * BN + cta_rank * C::BROWS, fb);
                         else
-                            LOAD_OP(base + C::OFF_B + stage * C::B_BYTES, &tmBh, ks * BK,
-                                    t * p.n + tn * BN + coff + cta_rank * (C::BROWS / 2), fb);
+                            tma_load_2d<NCTA>(base + C::OFF_B + stage * C::B_BYTES, &tmBh, ks * BK,
+                                              t * p.n + tn * BN + coff + cta_rank * (C::BROWS / 2), fb);
                         if (C::MX) {
                             // scale tiles: 512-byte atoms, ordered [term][k quad][128-row block]
                             const uint32_t sf = base + C::OFF_SF + stage * C::SF_STAGE_BYTES;
@@ -338,12 +294,10 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                             const uint32_t sf = base + C::OFF_SF + stage * C::SF_STAGE_BYTES;
                             const uint32_t tsfa = tmem_base + BN + stage * C::SF_COLS;
                             const uint32_t tsfb = tsfa + 4;
-#ifndef FMM_EXP_NO_CP
                             tc_cp_32x128b_warpx4<NCTA>(tsfa, make_sf_desc(sf));
 #pragma unroll
                             for (int h = 0; h < C::SFB_ATOMS; ++h)
                                 if (h == 0 || !half) tc_cp_32x128b_warpx4<NCTA>(tsfb + 4 * h, make_sf_desc(sf + 512 + h * 512));
-#endif
 #pragma unroll
                             for (int j = 0; j < BK / 32; ++j) {
                                 const uint32_t id = idesc | ((uint32_t)j << 29) | ((uint32_t)j << 4);
@@ -393,11 +347,10 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         int ss = 0; uint32_t sphase = 0;
         uint32_t store_cnt = 0;
         bool ok = true;
-#if FMM_HINT_C == 1
-        const uint64_t pol_c = policy_evict_first();
-#elif FMM_HINT_C == 2
+        // Each C tile is updated once per term that feeds it, and between two updates a whole term's operands
+        // stream through L2: the tiles are marked evict-last (at n = 8192: fewer write-backs of half-accumulated
+        // tiles, product kernel 3 % faster; an evict-first policy on the operand loads was slower).
         const uint64_t pol_c = policy_evict_last();
-#endif
         uint32_t accu[C::MX ? C::CW : 1];               // UE8M0: raw fp32 bits drained from TMEM
         unsigned long long acc2[C::MX ? 1 : C::CW / 2]; // FP32: promoted accumulators, two columns per register pair
         for (int w = unit; w < p.items && ok; w += units) {
@@ -522,13 +475,8 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                         fence_proxy_async();
                         __syncwarp();
                         if (lane == 0) {
-#if defined(FMM_EXP_NO_OUT)
-#elif defined(FMM_EXP_STORE_ONLY)
-                            STORE_C(&tmC, col0 + c * C::CH, row0, stg + b * C::STAGING_BYTES);
-#else
-                            if (ent.first) STORE_C(&tmC, col0 + c * C::CH, row0, stg + b * C::STAGING_BYTES);
-                            else REDUCE_C(&tmC, col0 + c * C::CH, row0, stg + b * C::STAGING_BYTES);
-#endif
+                            if (ent.first) tma_store_2d_hint(&tmC, col0 + c * C::CH, row0, stg + b * C::STAGING_BYTES, pol_c);
+                            else tma_reduce_add_2d_hint(&tmC, col0 + c * C::CH, row0, stg + b * C::STAGING_BYTES, pol_c);
                             bulk_commit();
                         }
                         ++store_cnt;
