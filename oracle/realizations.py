@@ -197,3 +197,28 @@ def rebalanced(U, V, W):
         Uo.append([float(x) / s for x in U[r]])
         Vo.append([float(x) * s for x in V[r]])
     return Uo, Vo, to_float(W)
+
+
+def _inv_t(M):
+    """Inverse transpose of a 2x2 matrix with rational (or float) entries."""
+    (a, b), (c, d) = M
+    det = a * d - b * c
+    return [[d / det, -c / det], [-b / det, a / det]]
+
+
+def _kron2(A, B):
+    """4x4 Kronecker product of two 2x2 matrices, rows/columns in the rv order (11, 12, 21, 22)."""
+    return [[A[i][j] * B[k][l] for j in range(2) for l in range(2)] for i in range(2) for k in range(2)]
+
+
+def _rowmat(rows, M):
+    return [[sum((r[j] * M[j][q] for j in range(4)), start=0 * r[0]) for q in range(4)] for r in rows]
+
+
+def act(U, V, W, X, Y, Z):
+    """Right action of (X, Y, Z) in GL_2^3 on a realization (Eq. A.1): u_r -> u_r (X (x) Y^-T),
+    v_r -> v_r (Y (x) Z^-T), w_r -> w_r (Z (x) X^-T) on the cyclic third factor.  Exact when the
+    coefficients are Q3 and the matrices hold Fractions; floating point otherwise."""
+    w = from_cyclic(W)          # the swap of entries 12 and 21 is its own inverse
+    return (_rowmat(U, _kron2(X, _inv_t(Y))), _rowmat(V, _kron2(Y, _inv_t(Z))),
+            from_cyclic(_rowmat(w, _kron2(Z, _inv_t(X)))))

@@ -67,10 +67,72 @@ def rebalanced(U, V, W):
     return U / s[:, None], V * s[:, None], W.copy()
 
 
+def phi(U, V, W):
+    """Phi = sum_r |U_r|^2 |V_r|^2 |W_r|^2 (Sec. 2.1)."""
+    U, V, W = (np.asarray(x, dtype=np.float64) for x in (U, V, W))
+    return float(np.sum((U ** 2).sum(1) * (V ** 2).sum(1) * (W ** 2).sum(1)))
+
+
+def act(U, V, W, X, Y, Z):
+    """Right action of g = (X, Y, Z) in GL_2^3 on a realization (Eq. A.1):
+    u_r -> u_r (X (x) Y^-T), v_r -> v_r (Y (x) Z^-T), w_r -> w_r (Z (x) X^-T), with w_r the cyclic third
+    factor rv(W_r^T), i.e. this library's W row with entries 12 and 21 swapped."""
+    it = lambda M: np.linalg.inv(M).T
+    cyc = [0, 2, 1, 3]
+    U2 = np.asarray(U, dtype=np.float64) @ np.kron(X, it(Y))
+    V2 = np.asarray(V, dtype=np.float64) @ np.kron(Y, it(Z))
+    w2 = np.asarray(W, dtype=np.float64)[:, cyc] @ np.kron(Z, it(X))
+    return U2, V2, w2[:, cyc]
+
+
+_DIRECTIONS = {"diag": np.array([[1.0, 0.0], [0.0, -1.0]]), "shear": np.array([[0.0, 1.0], [1.0, 0.0]])}
+
+
+def orbit_perturbation(factor, direction, sign, phi_target=24.0):
+    """A local perturbation of the Phi-optimal realization along one geodesic of the orbit (App. E.4):
+    T* . g with g = exp(sign * delta * H) in factor `factor` (0, 1, 2 = X, Y, Z), H = diag(1, -1) ("diag")
+    or [[0, 1], [1, 0]] ("shear"), and delta > 0 solved so that Phi = phi_target.  Phi is convex along the
+    geodesic with its minimum 200/9 at delta = 0 (Eq. A.2), so bisection on delta is enough.
+    Returns (U, V, W, delta) in float64, raw gauge."""
+    U, V, W = phi_optimal()
+    ev, Q = np.linalg.eigh(_DIRECTIONS[direction])
+
+    def arm(delta):
+        g = [np.eye(2), np.eye(2), np.eye(2)]
+        g[factor] = Q @ np.diag(np.exp(sign * delta * ev)) @ Q.T
+        return act(U, V, W, *g)
+
+    lo, hi = 0.0, 1.0
+    while phi(*arm(hi)) < phi_target:
+        hi *= 2.0
+    for _ in range(100):
+        mid = 0.5 * (lo + hi)
+        if phi(*arm(mid)) < phi_target:
+            lo = mid
+        else:
+            hi = mid
+    delta = 0.5 * (lo + hi)
+    return (*arm(delta), delta)
+
+
 NAMED = {"strassen": strassen, "winograd": winograd, "phi_optimal": phi_optimal, "cubic8": cubic8}
+PERTURBATIONS = [f"pert_f{f}_{d}_{s}" for f in range(3) for d in ("diag", "shear") for s in ("p", "m")]
+# the reconstructible part of the paper's fixed panel (Table E.2): three named arms and the twelve signed
+# perturbations at Phi = 24, all in the rebalanced gauge
+LADDER = ["phi_optimal_rb"] + [n + "_rb" for n in PERTURBATIONS] + ["strassen_rb", "winograd_rb"]
+
+
+def get64(name):
+    """float64 (U, V, W) of a named realization; `<name>_rb` = the same in the rebalanced gauge;
+    `pert_f<0|1|2>_<diag|shear>_<p|m>` = orbit_perturbation at Phi = 24."""
+    if name.endswith("_rb"):
+        return rebalanced(*get64(name[:-3]))
+    if name.startswith("pert_"):
+        _, f, d, s = name.split("_")
+        return orbit_perturbation(int(f[1]), d, +1 if s == "p" else -1)[:3]
+    return NAMED[name]()
 
 
 def get(name):
-    """fp32 (U, V, W) of a named realization."""
-    U, V, W = NAMED[name]()
-    return tuple(np.ascontiguousarray(x, dtype=np.float32) for x in (U, V, W))
+    """fp32 (U, V, W) of a named realization (see get64 for the names)."""
+    return tuple(np.ascontiguousarray(x, dtype=np.float32) for x in get64(name))

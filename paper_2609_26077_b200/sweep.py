@@ -5,6 +5,7 @@ emulated protocol, App. E.2), for the benchmark configurations.
     python -m paper_2609_26077_b200.sweep --config c1 [--scale-mode fp32|ue8m0] [--block-k 32|128]
                                           [--out sweep.jsonl] [--trials N]
     python -m paper_2609_26077_b200.sweep --summarise sweep.jsonl
+    python -m paper_2609_26077_b200.sweep --ladder sweep_c7.jsonl
 
 One JSON line is appended per (config, family, seed, realization, levels); on restart the keys that are
 already in the output file are skipped.  Everything is computed by the CUDA library (fmm_matmul,
@@ -23,8 +24,15 @@ import numpy as np
 
 from . import fmm, realizations as P, workloads as Wl
 
-PREDICTED = {"cubic": 1.0, "strassen": 2.0, "winograd": math.sqrt(7.0), "phi_optimal": 5.0 / 3.0}
 ALL = ["cubic", "strassen", "winograd", "phi_optimal"]
+
+
+def predicted(name, levels):
+    """sqrt(Phi/8)^levels: the model's RMS-constant ratio against the cubic product (Sec. 2.2, Sec. 3)."""
+    if name == "cubic":
+        return 1.0
+    return math.sqrt(P.phi(*P.get64(name)) / 8.0) ** max(levels, 1)
+
 
 # name -> (M, K, N), families, trials, realizations, levels
 CONFIGS = {
@@ -35,6 +43,10 @@ CONFIGS = {
     # operand-family controls (Sec. 4.3 / Table E.8): unit-variance families and Rademacher +-1 / +-10 cells
     "c6": dict(shape=(2048, 2048, 2048), families=["gaussian", "unit_uniform", "unit_laplace", "unit_t5", "rademacher", "rademacher10"],
                trials=8, names=ALL, levels=[1]),
+    # the reconstructible arms of the paper's fixed panel (Table E.2): optimum, twelve Phi = 24 perturbations,
+    # Strassen, Winograd form, all in the rebalanced gauge, on synthetic operands
+    "c7": dict(shape=(2048, 2048, 2048), families=["gaussian", "uniform", "llm"], trials=16,
+               names=["cubic"] + P.LADDER, levels=[1]),
     "c5": dict(shape=(2048, 2048, 2048), families=["scaled_gaussian", "student_t3"], trials=256, names=ALL, levels=[1, 2, 3]),
 }
 
@@ -110,12 +122,43 @@ def summarise(path, file=sys.stdout):
             cub = np.mean([cubic[s]["rel_frobenius"] for s in common]) if common else 0.0
             # operands the cubic product represents (almost) exactly make the ratio meaningless
             ratio = np.mean([seeds[s]["rel_frobenius"] for s in common]) / cub if cub > 1e-6 else float("nan")
-            pred = PREDICTED.get(name, float("nan")) ** max(lv, 1) if name != "cubic" else 1.0
+            pred = predicted(name, lv)
             rows.append((g, name, lv, len(e), e.mean(), e.std(), pooled, ratio, pred))
     print("| config | family | scales | blk | realization | levels | trials | mean rel. error | sd | pooled RMS | ratio vs cubic | sqrt(Phi/8)^l |", file=file)
     print("|---|---|---|---|---|---|---|---|---|---|---|---|", file=file)
     for g, name, lv, n, mean, sd, pooled, ratio, pred in rows:
         print(f"| {g[0]} | {g[1]} | {g[2]} | {g[3]} | {name} | {lv} | {n} | {mean:.5f} | {sd:.5f} | {pooled:.5f} | {ratio:.4f} | {pred:.4f} |", file=file)
+    return rows
+
+
+def ladder_summary(path, file=sys.stdout):
+    """Panel statistics of a c7 run, per (family, scale mode, block): Spearman correlation between Phi and the
+    mean error over the arms, the fraction of trials on which the optimum beats all twelve perturbations at
+    once, and the relative gap between the optimum and the best arm (the paper's O2 / panel-gap statistics,
+    here on synthetic operands)."""
+    recs = [json.loads(line) for line in open(path) if line.strip()]
+    groups = defaultdict(lambda: defaultdict(dict))
+    for r in recs:
+        if r["realization"] != "cubic":
+            groups[(r["family"], r["scale_mode"], r["block_k"])][r["realization"]][r["seed"]] = r["rel_frobenius"]
+    rows = []
+    for g, by in sorted(groups.items()):
+        arms = [a for a in P.LADDER if a in by]
+        seeds = sorted(set.intersection(*[set(by[a]) for a in arms]))
+        mean = np.array([np.mean([by[a][s] for s in seeds]) for a in arms])
+        phis = np.array([P.phi(*P.get64(a)) for a in arms])
+        rk = lambda x: np.argsort(np.argsort(x, kind="stable"), kind="stable").astype(float)
+        # ties in Phi (the twelve arms at 24) get their average rank
+        rphi = np.array([np.mean(rk(phis)[phis == v]) for v in phis])
+        rho = float(np.corrcoef(rphi, rk(mean))[0, 1])
+        perts = [a for a in arms if a.startswith("pert_")]
+        wins = np.mean([all(by["phi_optimal_rb"][s] < by[a][s] for a in perts) for s in seeds])
+        gap = float(mean[arms.index("phi_optimal_rb")] / mean.min() - 1.0)
+        rows.append((g, len(seeds), rho, float(wins), gap, arms[int(mean.argmin())]))
+    print("| family | scales | blk | trials | Spearman(Phi, mean error) | optimum beats all 12 perturbations | panel gap | best arm |", file=file)
+    print("|---|---|---|---|---|---|---|---|", file=file)
+    for g, n, rho, wins, gap, best in rows:
+        print(f"| {g[0]} | {g[1]} | {g[2]} | {n} | {rho:.3f} | {wins:.3f} | {gap:.4f} | {best} |", file=file)
     return rows
 
 
@@ -127,9 +170,12 @@ def main():
     ap.add_argument("--out", default="sweep.jsonl")
     ap.add_argument("--trials", type=int, default=0)
     ap.add_argument("--summarise")
+    ap.add_argument("--ladder", help="panel statistics of a c7 output file")
     a = ap.parse_args()
     if a.summarise:
         summarise(a.summarise)
+    elif a.ladder:
+        ladder_summary(a.ladder)
     else:
         if not a.config:
             ap.error("--config or --summarise is required")
