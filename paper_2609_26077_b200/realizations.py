@@ -115,21 +115,42 @@ def orbit_perturbation(factor, direction, sign, phi_target=24.0):
     return (*arm(delta), delta)
 
 
+def orbit_member(k, spread=0.25):
+    """Member k of a seeded family of exact orbit points T* . g_k (App. E.8, orbit-ratio stability): in each
+    factor g = exp(S) R with S a random symmetric traceless matrix of norm <= spread and R a random rotation,
+    so the members differ in Phi as well as in frame.  Member 0 is T* itself."""
+    U, V, W = phi_optimal()
+    if k == 0:
+        return U, V, W
+    rng = np.random.default_rng([2609, 26077, k])
+    g = []
+    for _ in range(3):
+        a, b = rng.uniform(-spread, spread, 2) / math.sqrt(2.0)
+        ev, Q = np.linalg.eigh(np.array([[a, b], [b, -a]]))
+        th = rng.uniform(0.0, 2.0 * math.pi)
+        R = np.array([[math.cos(th), -math.sin(th)], [math.sin(th), math.cos(th)]])
+        g.append(Q @ np.diag(np.exp(ev)) @ Q.T @ R)
+    return act(U, V, W, *g)
+
+
 NAMED = {"strassen": strassen, "winograd": winograd, "phi_optimal": phi_optimal, "cubic8": cubic8}
 PERTURBATIONS = [f"pert_f{f}_{d}_{s}" for f in range(3) for d in ("diag", "shear") for s in ("p", "m")]
 # the reconstructible part of the paper's fixed panel (Table E.2): three named arms and the twelve signed
 # perturbations at Phi = 24, all in the rebalanced gauge
+ORBIT15 = [f"orbit_{k:02d}_rb" for k in range(15)]
 LADDER = ["phi_optimal_rb"] + [n + "_rb" for n in PERTURBATIONS] + ["strassen_rb", "winograd_rb"]
 
 
 def get64(name):
     """float64 (U, V, W) of a named realization; `<name>_rb` = the same in the rebalanced gauge;
-    `pert_f<0|1|2>_<diag|shear>_<p|m>` = orbit_perturbation at Phi = 24."""
+    `pert_f<0|1|2>_<diag|shear>_<p|m>` = orbit_perturbation at Phi = 24; `orbit_<k>` = orbit_member(k)."""
     if name.endswith("_rb"):
         return rebalanced(*get64(name[:-3]))
     if name.startswith("pert_"):
         _, f, d, s = name.split("_")
         return orbit_perturbation(int(f[1]), d, +1 if s == "p" else -1)[:3]
+    if name.startswith("orbit_"):
+        return orbit_member(int(name.split("_")[1]))
     return NAMED[name]()
 
 

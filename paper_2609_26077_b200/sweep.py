@@ -47,6 +47,8 @@ CONFIGS = {
     # Strassen, Winograd form, all in the rebalanced gauge, on synthetic operands
     "c7": dict(shape=(2048, 2048, 2048), families=["gaussian", "uniform", "llm"], trials=16,
                names=["cubic"] + P.LADDER, levels=[1]),
+    # orbit-ratio stability (Table E.8): fifteen exact orbit members, one shape, signed-uniform operands
+    "c8": dict(shape=(2048, 2048, 2048), families=["uniform"], trials=8, names=["cubic"] + P.ORBIT15, levels=[1]),
     "c5": dict(shape=(2048, 2048, 2048), families=["scaled_gaussian", "student_t3"], trials=256, names=ALL, levels=[1, 2, 3]),
 }
 
@@ -162,6 +164,22 @@ def ladder_summary(path, file=sys.stdout):
     return rows
 
 
+def orbit_stability(path, file=sys.stdout):
+    """Coefficient of variation, over the orbit members of a c8 run, of (measured error ratio against cubic) /
+    sqrt(Phi/8): how stable the model's one free constant is along the orbit (Table E.8 reports 0.37 %)."""
+    rows = [r for r in summarise(path, file=open(os.devnull, "w")) if r[1].startswith("orbit_")]
+    out = []
+    for g in sorted(set(r[0] for r in rows)):
+        q = np.array([r[7] / r[8] for r in rows if r[0] == g])
+        phis = np.array([r[8] ** 2 * 8 for r in rows if r[0] == g])
+        out.append((g, len(q), float(phis.min()), float(phis.max()), float(q.mean()), float(q.std(ddof=1) / q.mean())))
+    print("| family | scales | blk | members | Phi range | mean measured/predicted | CV |", file=file)
+    print("|---|---|---|---|---|---|---|", file=file)
+    for g, n, lo, hi, m, cv in out:
+        print(f"| {g[1]} | {g[2]} | {g[3]} | {n} | {lo:.2f} - {hi:.2f} | {m:.4f} | {100 * cv:.2f} % |", file=file)
+    return out
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--config", choices=sorted(CONFIGS))
@@ -171,11 +189,14 @@ def main():
     ap.add_argument("--trials", type=int, default=0)
     ap.add_argument("--summarise")
     ap.add_argument("--ladder", help="panel statistics of a c7 output file")
+    ap.add_argument("--orbit", help="orbit-ratio stability of a c8 output file")
     a = ap.parse_args()
     if a.summarise:
         summarise(a.summarise)
     elif a.ladder:
         ladder_summary(a.ladder)
+    elif a.orbit:
+        orbit_stability(a.orbit)
     else:
         if not a.config:
             ap.error("--config or --summarise is required")

@@ -116,3 +116,16 @@ def test_ladder_is_ordered_by_phi():
     phis = [P.phi(*P.get64(n)) for n in P.LADDER]
     assert all(b >= a - 1e-9 for a, b in zip(phis, phis[1:]))
     assert abs(phis[0] - 200.0 / 9.0) < 1e-12 and abs(phis[-2] - 32.0) < 1e-12 and abs(phis[-1] - 56.0) < 1e-12
+
+
+def test_orbit_members_are_exact_algorithms_with_phi_above_the_minimum():
+    # every member of the orbit satisfies the Brent equations and has Phi >= 200/9 (the certificate, Sec. 3)
+    phis = []
+    for name in P.ORBIT15:
+        U, V, W = P.get64(name)
+        res = R.brent_residuals(*[[[float(x) for x in r] for r in M] for M in (U, V, W)])
+        assert max(abs(float(x)) for x in res) < 1e-12
+        phis.append(P.phi(U, V, W))
+    assert abs(phis[0] - 200.0 / 9.0) < 1e-12
+    assert all(p > 200.0 / 9.0 + 1e-6 for p in phis[1:])
+    assert max(phis) > 28.0          # the family spans a range of Phi, not just frames
