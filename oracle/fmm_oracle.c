@@ -110,6 +110,8 @@ typedef struct {
     int blk;          /* block length along the contracted axis */
     int mode;         /* SCALE_FP32 | SCALE_UE8M0 | SCALE_IDENTITY */
     float amax_floor; /* minimum-scale clamp, 1e-12 in the paper */
+    int b_tile;       /* 0, or the width of the weight-side scale tiles (blk x b_tile, App. E.5) */
+    int b_bf16;       /* nonzero: round each encoded weight combination to bf16 before quantizing */
 } qparams_t;
 
 /* Quantize one block of `blk` values x[0], x[stride], ...  Writes the codes with
@@ -164,7 +166,7 @@ void oracle_quant_rows(const float *X, int64_t rows, int64_t cols, int64_t ld,
                        int blk, int mode, float amax_floor,
                        uint8_t *codes, float *scales, uint8_t *e8)
 {
-    qparams_t qp = { blk, mode, amax_floor };
+    qparams_t qp = { blk, mode, amax_floor, 0, 0 };
     int64_t nb = cols / blk;
     for (int64_t i = 0; i < rows; ++i)
         for (int64_t b = 0; b < nb; ++b)
@@ -179,13 +181,67 @@ void oracle_quant_cols(const float *X, int64_t rows, int64_t cols, int64_t ld,
                        int blk, int mode, float amax_floor,
                        uint8_t *codes, float *scales, uint8_t *e8)
 {
-    qparams_t qp = { blk, mode, amax_floor };
+    qparams_t qp = { blk, mode, amax_floor, 0, 0 };
     int64_t nb = rows / blk;
     for (int64_t b = 0; b < nb; ++b)
         for (int64_t j = 0; j < cols; ++j)
             scales[b * cols + j] = quant_block(X + b * blk * ld + j, ld, blk, &qp,
                                                codes + b * blk * cols + j, cols,
                                                e8 ? e8 + b * cols + j : NULL);
+}
+
+/* B side, deployment-matched grouping (App. E.5): one scale per tile of blk x tile entries, the maximum
+ * taken over the whole tile of the (already encoded) operand.  FP32 scales only.  The scale is written
+ * for every column of the tile, so the output shapes are those of oracle_quant_cols. */
+void oracle_quant_tiles(const float *X, int64_t rows, int64_t cols, int64_t ld,
+                        int blk, int tile, float amax_floor,
+                        uint8_t *codes, float *scales)
+{
+    int64_t nb = rows / blk;
+    for (int64_t b = 0; b < nb; ++b)
+        for (int64_t j0 = 0; j0 < cols; j0 += tile) {
+            int64_t j1 = j0 + tile < cols ? j0 + tile : cols;
+            float amax = 0.0f;
+            for (int64_t i = 0; i < blk; ++i)
+                for (int64_t j = j0; j < j1; ++j) {
+                    float a = fabsf(X[(b * blk + i) * ld + j]);
+                    if (a > amax) amax = a;
+                }
+            float amax_c = amax > amax_floor ? amax : amax_floor;
+            float s = amax_c / 448.0f;
+            float inv = 448.0f / amax_c;
+            for (int64_t i = 0; i < blk; ++i)
+                for (int64_t j = j0; j < j1; ++j)
+                    codes[(b * blk + i) * cols + j] = oracle_e4m3_encode(X[(b * blk + i) * ld + j] * inv);
+            for (int64_t j = j0; j < j1; ++j) scales[b * cols + j] = s;
+        }
+}
+
+/* Round to bfloat16 (8 significant bits), nearest even, result widened back to fp32. */
+float oracle_bf16_round(float x)
+{
+    uint32_t u = f32_bits(x);
+    if ((u & 0x7f800000u) == 0x7f800000u) return x;          /* inf / nan unchanged */
+    u += 0x7fffu + ((u >> 16) & 1u);
+    return bits_f32(u & 0xffff0000u);
+}
+
+/* Weight-side leaf quantizer with the optional deployment-matched steps. */
+static void quant_b_leaf(const float *X, int64_t rows, int64_t cols, int64_t ld, const qparams_t *qp,
+                         uint8_t *codes, float *scales, uint8_t *e8)
+{
+    const float *src = X;
+    int64_t sld = ld;
+    float *tmp = NULL;
+    if (qp->b_bf16) {
+        tmp = (float *)malloc(sizeof(float) * rows * cols);
+        for (int64_t i = 0; i < rows; ++i)
+            for (int64_t j = 0; j < cols; ++j) tmp[i * cols + j] = oracle_bf16_round(X[i * ld + j]);
+        src = tmp; sld = cols;
+    }
+    if (qp->b_tile) oracle_quant_tiles(src, rows, cols, sld, qp->blk, qp->b_tile, qp->amax_floor, codes, scales);
+    else oracle_quant_cols(src, rows, cols, sld, qp->blk, qp->mode, qp->amax_floor, codes, scales, e8);
+    free(tmp);
 }
 
 /* -------------------------------------------------- linear combinations */
@@ -290,7 +346,7 @@ static void leaf_product(const float *A, int64_t lda, const float *B, int64_t ld
         uint8_t *cb = (uint8_t *)malloc((size_t)(k * n));
         float *sb = (float *)malloc(sizeof(float) * nb * n);
         oracle_quant_rows(A, m, k, lda, qp->blk, qp->mode, qp->amax_floor, ca, sa, NULL);
-        oracle_quant_cols(B, k, n, ldb, qp->blk, qp->mode, qp->amax_floor, cb, sb, NULL);
+        quant_b_leaf(B, k, n, ldb, qp, cb, sb, NULL);
         for (int64_t i = 0; i < m; ++i)
             for (int64_t p = 0; p < k; ++p)
                 Ad[i * k + p] = oracle_e4m3_decode(ca[i * k + p]) * (double)sa[i * nb + p / qp->blk];
@@ -350,6 +406,7 @@ static void fill_realization(realization_t *D, int rank, const float *U, const f
             D->W[r][j] = W ? W[r * 4 + j] : 0.0f;
         }
     D->qp.blk = blk; D->qp.mode = mode; D->qp.amax_floor = amax_floor;
+    D->qp.b_tile = 0; D->qp.b_bf16 = 0;
 }
 
 /* C (fp64, M x N) = fused block-scaled fast product of A (M x K) and B (K x N).
@@ -369,6 +426,25 @@ int oracle_fused_fmm(const float *A, const float *B, double *C,
     return 0;
 }
 
+/* Same, with the weight-side options of App. E.5: b_tile = 0 or the tile width of the weight scales
+ * (FP32 scales, blk x b_tile tiles), b_bf16 != 0 rounds each encoded weight combination to bf16 first. */
+int oracle_fused_fmm_ex(const float *A, const float *B, double *C,
+                        int64_t M, int64_t N, int64_t K,
+                        int rank, const float *U, const float *V, const float *W,
+                        int levels, int blk, int mode, float amax_floor, int b_tile, int b_bf16)
+{
+    if (rank > ORACLE_MAX_RANK || levels < 0) return 1;
+    int64_t div = (int64_t)1 << levels;
+    if (M % div || N % div || K % div) return 2;
+    if (mode != SCALE_IDENTITY && (K / div) % blk) return 3;
+    if (b_tile && (mode != SCALE_FP32 || (N / div) % b_tile)) return 4;
+    realization_t D;
+    fill_realization(&D, rank, U, V, W, blk, mode, amax_floor);
+    D.qp.b_tile = b_tile; D.qp.b_bf16 = b_bf16;
+    fused_rec(&D, levels, A, K, B, N, M, N, K, C);
+    return 0;
+}
+
 /* ------------------------------- quantized leaf operands, for bit parity */
 
 static void encode_rec(const realization_t *D, int levels, int side,
@@ -382,7 +458,7 @@ static void encode_rec(const realization_t *D, int levels, int side,
         float *s = scales + *term * nsc;
         uint8_t *e = e8 ? e8 + *term * nsc : NULL;
         if (side == 0) oracle_quant_rows(X, rows, cols, ld, D->qp.blk, D->qp.mode, D->qp.amax_floor, c, s, e);
-        else           oracle_quant_cols(X, rows, cols, ld, D->qp.blk, D->qp.mode, D->qp.amax_floor, c, s, e);
+        else           quant_b_leaf(X, rows, cols, ld, &D->qp, c, s, e);
         *term += 1;
         return;
     }
@@ -410,6 +486,24 @@ int oracle_encode(const float *X, int64_t rows, int64_t cols, int side,
     if (((side == 0 ? cols : rows) / div) % blk) return 3;
     realization_t D;
     fill_realization(&D, rank, U, V, NULL, blk, mode, amax_floor);
+    int64_t term = 0;
+    encode_rec(&D, levels, side, X, cols, rows, cols, &term, codes, scales, e8);
+    return 0;
+}
+
+int oracle_encode_ex(const float *X, int64_t rows, int64_t cols, int side,
+                     int rank, const float *U, const float *V,
+                     int levels, int blk, int mode, float amax_floor, int b_tile, int b_bf16,
+                     uint8_t *codes, float *scales, uint8_t *e8)
+{
+    if (rank > ORACLE_MAX_RANK || levels < 0 || mode == SCALE_IDENTITY) return 1;
+    int64_t div = (int64_t)1 << levels;
+    if (rows % div || cols % div) return 2;
+    if (((side == 0 ? cols : rows) / div) % blk) return 3;
+    if (b_tile && (mode != SCALE_FP32 || (side == 1 && (cols / div) % b_tile))) return 4;
+    realization_t D;
+    fill_realization(&D, rank, U, V, NULL, blk, mode, amax_floor);
+    D.qp.b_tile = b_tile; D.qp.b_bf16 = b_bf16;
     int64_t term = 0;
     encode_rec(&D, levels, side, X, cols, rows, cols, &term, codes, scales, e8);
     return 0;

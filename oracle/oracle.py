@@ -29,6 +29,10 @@ def lib():
         L.oracle_e4m3_decode.argtypes = [C.c_uint8]
         L.oracle_fused_fmm.restype = C.c_int
         L.oracle_encode.restype = C.c_int
+        L.oracle_fused_fmm_ex.restype = C.c_int
+        L.oracle_encode_ex.restype = C.c_int
+        L.oracle_bf16_round.restype = C.c_float
+        L.oracle_bf16_round.argtypes = [C.c_float]
         L.oracle_num_threads.restype = C.c_int
         _lib = L
     return _lib
@@ -90,6 +94,24 @@ def quant_cols(X, blk, mode=SCALE_FP32, amax_floor=AMAX_FLOOR):
     return codes, scales, e8
 
 
+def quant_tiles(X, blk, tile, amax_floor=AMAX_FLOOR):
+    """B-side quantizer with one FP32 scale per blk x tile tile (App. E.5); shapes as quant_cols."""
+    X = _f32(X)
+    rows, cols = X.shape
+    codes = np.empty((rows, cols), np.uint8)
+    scales = np.empty((rows // blk, cols), np.float32)
+    lib().oracle_quant_tiles(_p(X), C.c_int64(rows), C.c_int64(cols), C.c_int64(cols), C.c_int(blk), C.c_int(tile),
+                             C.c_float(float(amax_floor)), _p(codes), _p(scales))
+    return codes, scales
+
+
+def bf16_round(x):
+    """Elementwise round-to-nearest-even to bfloat16, widened back to fp32."""
+    x = _f32(np.atleast_1d(x))
+    f = lib().oracle_bf16_round
+    return np.array([f(float(v)) for v in x.ravel()], np.float32).reshape(x.shape)
+
+
 def _uvw(U, V, W):
     U = _f32(U) if U is not None else None
     V = _f32(V) if V is not None else None
@@ -98,8 +120,9 @@ def _uvw(U, V, W):
 
 
 def fused_fmm(A, B, U=None, V=None, W=None, levels=1, blk=32, mode=SCALE_FP32,
-              amax_floor=AMAX_FLOOR):
-    """C (fp64) of the fused block-scaled fast product; levels=0 is cubic fp8."""
+              amax_floor=AMAX_FLOOR, b_tile=0, b_bf16=False):
+    """C (fp64) of the fused block-scaled fast product; levels=0 is cubic fp8.
+    b_tile / b_bf16: the weight-side options of App. E.5 (blk x b_tile scale tiles, bf16 pre-round)."""
     A, B = _f32(A), _f32(B)
     M, K = A.shape
     K2, N = B.shape
@@ -107,17 +130,17 @@ def fused_fmm(A, B, U=None, V=None, W=None, levels=1, blk=32, mode=SCALE_FP32,
     U, V, W = _uvw(U, V, W)
     rank = 0 if U is None else U.shape[0]
     Cout = np.empty((M, N), np.float64)
-    rc = lib().oracle_fused_fmm(_p(A), _p(B), _p(Cout), C.c_int64(M), C.c_int64(N), C.c_int64(K),
-                                C.c_int(rank), _p(U) if U is not None else None,
-                                _p(V) if V is not None else None, _p(W) if W is not None else None,
-                                C.c_int(levels), C.c_int(blk), C.c_int(mode),
-                                C.c_float(float(amax_floor)))
+    rc = lib().oracle_fused_fmm_ex(_p(A), _p(B), _p(Cout), C.c_int64(M), C.c_int64(N), C.c_int64(K),
+                                   C.c_int(rank), _p(U) if U is not None else None,
+                                   _p(V) if V is not None else None, _p(W) if W is not None else None,
+                                   C.c_int(levels), C.c_int(blk), C.c_int(mode),
+                                   C.c_float(float(amax_floor)), C.c_int(int(b_tile)), C.c_int(int(bool(b_bf16))))
     if rc:
         raise ValueError(f"oracle_fused_fmm rejected the arguments (code {rc})")
     return Cout
 
 
-def encode(X, side, U, V, levels, blk=32, mode=SCALE_FP32, amax_floor=AMAX_FLOOR):
+def encode(X, side, U, V, levels, blk=32, mode=SCALE_FP32, amax_floor=AMAX_FLOOR, b_tile=0, b_bf16=False):
     """Quantized leaf operands of one side ('A' or 'B'), depth-first term order.
     'A': codes [T, m, k], scales [T, m, k/blk];  'B': codes [T, k, n], scales [T, k/blk, n]."""
     X = _f32(X)
@@ -132,10 +155,11 @@ def encode(X, side, U, V, levels, blk=32, mode=SCALE_FP32, amax_floor=AMAX_FLOOR
     sshape = (T, lr, lc // blk) if s == 0 else (T, lr // blk, lc)
     scales = np.empty(sshape, np.float32)
     e8 = np.empty(sshape, np.uint8)
-    rc = lib().oracle_encode(_p(X), C.c_int64(rows), C.c_int64(cols), C.c_int(s), C.c_int(rank),
-                             _p(U) if U is not None else None, _p(V) if V is not None else None,
-                             C.c_int(levels), C.c_int(blk), C.c_int(mode),
-                             C.c_float(float(amax_floor)), _p(codes), _p(scales), _p(e8))
+    rc = lib().oracle_encode_ex(_p(X), C.c_int64(rows), C.c_int64(cols), C.c_int(s), C.c_int(rank),
+                                _p(U) if U is not None else None, _p(V) if V is not None else None,
+                                C.c_int(levels), C.c_int(blk), C.c_int(mode),
+                                C.c_float(float(amax_floor)), C.c_int(int(b_tile)), C.c_int(int(bool(b_bf16))),
+                                _p(codes), _p(scales), _p(e8))
     if rc:
         raise ValueError(f"oracle_encode rejected the arguments (code {rc})")
     return codes, scales, e8
