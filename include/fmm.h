@@ -62,6 +62,15 @@ typedef struct {
     fmm_scale_mode_t scale_mode;
     float amax_floor;            /* minimum-scale clamp on the block amax; the paper uses 1e-12 */
     float fp8_max;               /* largest e4m3 magnitude; must be 448 */
+    /* Deployment-matched weight-side options (App. E.5; both 0 for the paper's emulated protocol):
+     * b_tile_n = 128 takes one scale per tile of 128 k x 128 columns of each encoded B-side
+     * combination (the maximum is taken after the combination is formed), instead of one per column
+     * and block; requires block_k == 128, FMM_SCALE_FP32_AMAX_DIV_448 and a leaf N divisible by 128.
+     * b_preround_bf16 != 0 rounds each encoded B-side combination to bfloat16 (nearest even) before
+     * the maximum and the e4m3 cast; same requirements on block_k and scale_mode.  The scale array keeps its shape: every column of a tile
+     * carries the tile's scale. */
+    int b_tile_n;
+    int b_preround_bf16;
 } fmm_quant_params_t;
 
 typedef struct fmm_plan fmm_plan_t;   /* opaque */

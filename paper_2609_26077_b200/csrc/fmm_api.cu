@@ -102,13 +102,15 @@ fmm_status_t encode_side(fmm_plan* plan, const FmmLayout& L, char* ws, const flo
     e.s_out = ws + (b_side ? L.sb : L.sa);
     e.s_term_stride = (int64_t)(b_side ? L.sb_term : L.sa_term);
     e.amax_floor = plan->qp.amax_floor;
+    e.b_tile = b_side ? plan->qp.b_tile_n : 0;
+    e.preround_bf16 = (b_side && plan->qp.b_preround_bf16) ? 1 : 0;
     fmm_status_t s;
     if (lv == 0) {
         // Plain quantization of the matrix itself.  The matrix is cut into four panels (row panels of A,
         // column panels of B) that are handled like four "combinations" with identity coefficients, so
         // each thread keeps four independent loads in flight; the outputs land where the unsplit
         // matrix would put them.
-        const bool panels = b_side ? (cols % 256 == 0) : (rows % 4 == 0);
+        const bool panels = b_side ? (cols % (e.b_tile ? 512 : 256) == 0) : (rows % 4 == 0);
         e.in = X; e.in_batch_stride = 0; e.ld = cols; e.batch = 1;
         if (panels) {
             e.nq = 4; e.R = 4;
@@ -255,6 +257,9 @@ fmm_status_t fmm_plan_create(fmm_plan_t** out, int rank, const float* U, const f
     if (qp->scale_mode != FMM_SCALE_FP32_AMAX_DIV_448 && qp->scale_mode != FMM_SCALE_UE8M0_CEIL) return FMM_ERR_INVALID_ARG;
     if (qp->scale_mode == FMM_SCALE_UE8M0_CEIL && qp->block_k != 32) return FMM_ERR_INVALID_ARG;
     if (qp->fp8_max != 448.0f || !(qp->amax_floor > 0.0f) || !isfinite(qp->amax_floor)) return FMM_ERR_INVALID_ARG;
+    if (qp->b_tile_n != 0 && qp->b_tile_n != 128) return FMM_ERR_INVALID_ARG;
+    if ((qp->b_tile_n == 128 || qp->b_preround_bf16) &&
+        (qp->block_k != 128 || qp->scale_mode != FMM_SCALE_FP32_AMAX_DIV_448)) return FMM_ERR_INVALID_ARG;
     if (levels > 0) {
         if (rank < 1 || rank > FMM_MAX_RANK || !U || !V || !W) return FMM_ERR_INVALID_ARG;
         if (!finite_all(U, rank * 4) || !finite_all(V, rank * 4) || !finite_all(W, rank * 4)) return FMM_ERR_INVALID_ARG;

@@ -10,6 +10,7 @@
 //
 // Both kernels are HBM-bound streaming kernels: every input element is read once with
 // full-line coalesced loads and every output byte is written once in whole 32-byte sectors.
+#include <cuda_bf16.h>
 #include "fmm_internal.h"
 #include "fmm_ptx.cuh"
 
@@ -202,6 +203,12 @@ __global__ void __launch_bounds__(256) encode_a_kernel(const EncodeParams p)
 // is two 64-byte row segments per warp; each thread writes 16 contiguous code bytes and the two
 // lanes of a block fill one 32-byte sector.  BLK == 128 takes a second pass over the four
 // 32-element sub-blocks (served by L1/L2).
+//
+// TILE (App. E.5, the deployment-matched weight grouping; BLK == 128, FP32 scales): one scale per tile of
+// 128 k x 128 columns of each encoded combination.  A block of 256 threads then covers a whole tile, the
+// column maxima of the first pass are reduced across the block, and every column stores the tile's scale,
+// so the scale array keeps its per-column shape.  p.preround_bf16 rounds each encoded combination to
+// bfloat16 (nearest even) before the maximum and the cast, as the paper's real kernel does.
 template <int MODE>
 __device__ __forceinline__ void store_b_scale(const EncodeParams& p, int64_t t, int r, int j, int kb, int kc,
                                               float s, uint32_t e8word, bool last_of_word)
@@ -216,13 +223,16 @@ __device__ __forceinline__ void store_b_scale(const EncodeParams& p, int64_t t, 
     }
 }
 
-template <int BLK, int MODE, uint32_t NZ>
-__global__ void __launch_bounds__(128, 4) encode_b_kernel(const EncodeParams p)
+template <int BLK, int MODE, uint32_t NZ, bool TILE, bool PRE>
+__global__ void __launch_bounds__(TILE ? 256 : 128, TILE ? 2 : 4) encode_b_kernel(const EncodeParams p)
 {
+    static_assert(!(TILE || PRE) || (BLK == 128 && MODE == FMM_SCALE_FP32_AMAX_DIV_448), "weight-side options: blk 128, fp32");
     // here p.rows = leaf k (contracted), p.cols = leaf n
     constexpr unsigned FULL = 0xffffffffu;
+    constexpr int WARPS = TILE ? 8 : 4;
+    __shared__ float tile_amax[TILE ? WARPS : 1][FMM_MAX_RANK];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int j = blockIdx.x * 64 + warp * 16 + (lane & 15);
+    const int j = blockIdx.x * (WARPS * 16) + warp * 16 + (lane & 15);
     const int khalf = lane >> 4;
     const int kc = blockIdx.y;                      // chunk of 128 k
     const int b = blockIdx.z;
@@ -271,6 +281,10 @@ __global__ void __launch_bounds__(128, 4) encode_b_kernel(const EncodeParams p)
 #pragma unroll
                         for (int kk = 0; kk < 16; ++kk) v[kk] = 0.0f;
                     }
+                    if (PRE) {
+#pragma unroll
+                        for (int kk = 0; kk < 16; ++kk) v[kk] = __bfloat162float(__float2bfloat16_rn(v[kk]));
+                    }
                     const int64_t t = (int64_t)b * p.R + r;
                     if (BLK == 32 || pass == 0) {
                         float amax = 0.0f;
@@ -279,7 +293,7 @@ __global__ void __launch_bounds__(128, 4) encode_b_kernel(const EncodeParams p)
                         amax = fmaxf(amax, __shfl_xor_sync(FULL, amax, 16));
                         if (BLK == 32) blk_amax[r] = amax; else blk_amax[r] = fmaxf(blk_amax[r], amax);
                     }
-                    if (BLK == 32 || (pass == 0 && sub == 3)) {
+                    if (!TILE && (BLK == 32 || (pass == 0 && sub == 3))) {
                         float sc; uint32_t e8;
                         blk_inv[r] = block_scale<MODE>(blk_amax[r], p.amax_floor, sc, e8);
                         const int kb = (BLK == 32) ? (kc * 4 + sub) : kc;
@@ -296,6 +310,28 @@ __global__ void __launch_bounds__(128, 4) encode_b_kernel(const EncodeParams p)
                         *reinterpret_cast<uint4*>(p.q_out + t * term_codes + (int64_t)j * p.rows + k0) =
                             make_uint4(wv[0], wv[1], wv[2], wv[3]);
                     }
+                }
+            }
+        }
+        if (TILE && pass == 0) {
+            // column maxima -> tile maximum: 16 columns per warp by shuffles, 8 warps through shared memory
+#pragma unroll
+            for (int r = 0; r < FMM_MAX_RANK; ++r) {
+                float a = blk_amax[r];
+#pragma unroll
+                for (int d = 8; d >= 1; d >>= 1) a = fmaxf(a, __shfl_xor_sync(FULL, a, d));
+                if (lane == 0) tile_amax[warp][r] = a;
+            }
+            __syncthreads();
+#pragma unroll
+            for (int r = 0; r < FMM_MAX_RANK; ++r) {
+                if (row_used<NZ>(r, p.R)) {
+                    float a = tile_amax[0][r];
+#pragma unroll
+                    for (int w = 1; w < WARPS; ++w) a = fmaxf(a, tile_amax[w][r]);
+                    float sc; uint32_t e8;
+                    blk_inv[r] = block_scale<MODE>(a, p.amax_floor, sc, e8);
+                    if (khalf == 0) store_b_scale<MODE>(p, (int64_t)b * p.R + r, r, j, kc, kc, sc, 0u, false);
                 }
             }
         }
@@ -447,10 +483,24 @@ void launch_b(const EncodeParams& p, dim3 grid, cudaStream_t st)
 {
     const uint32_t m = (p.nq == 4) ? coef_mask(p) : 0u;
     switch (m) {
-#define X(M) case M: encode_b_kernel<BLK, MODE, M><<<grid, 128, 0, st>>>(p); return;
+#define X(M) case M: encode_b_kernel<BLK, MODE, M, false, false><<<grid, 128, 0, st>>>(p); return;
         FMM_KNOWN_MASKS(X)
 #undef X
-        default: encode_b_kernel<BLK, MODE, 0u><<<grid, 128, 0, st>>>(p); return;
+        default: encode_b_kernel<BLK, MODE, 0u, false, false><<<grid, 128, 0, st>>>(p); return;
+    }
+}
+// weight-side options (tile scales and / or bf16 pre-round): blk 128, fp32 scales
+template <bool TILE, bool PRE>
+void launch_b_opt(const EncodeParams& p, dim3 grid, cudaStream_t st)
+{
+    constexpr int F = FMM_SCALE_FP32_AMAX_DIV_448;
+    constexpr int T = TILE ? 256 : 128;
+    const uint32_t m = (p.nq == 4) ? coef_mask(p) : 0u;
+    switch (m) {
+#define X(M) case M: encode_b_kernel<128, F, M, TILE, PRE><<<grid, T, 0, st>>>(p); return;
+        FMM_KNOWN_MASKS(X)
+#undef X
+        default: encode_b_kernel<128, F, 0u, TILE, PRE><<<grid, T, 0, st>>>(p); return;
     }
 }
 }  // namespace
@@ -476,7 +526,12 @@ fmm_status_t fmm_launch_encode_a(const EncodeParams& p, int blk, int mode, cudaS
 fmm_status_t fmm_launch_encode_b(const EncodeParams& p, int blk, int mode, cudaStream_t st)
 {
     dim3 grid((unsigned)(p.cols / 64), (unsigned)(p.rows / 128), (unsigned)p.batch);
-    if (mode == FMM_SCALE_FP32_AMAX_DIV_448) {
+    if (p.b_tile || p.preround_bf16) {
+        if (p.b_tile) grid.x = (unsigned)(p.cols / 128);
+        if (p.b_tile && p.preround_bf16) launch_b_opt<true, true>(p, grid, st);
+        else if (p.b_tile) launch_b_opt<true, false>(p, grid, st);
+        else launch_b_opt<false, true>(p, grid, st);
+    } else if (mode == FMM_SCALE_FP32_AMAX_DIV_448) {
         if (blk == 32) launch_b<32, FMM_SCALE_FP32_AMAX_DIV_448>(p, grid, st);
         else launch_b<128, FMM_SCALE_FP32_AMAX_DIV_448>(p, grid, st);
     } else {

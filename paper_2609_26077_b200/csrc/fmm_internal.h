@@ -59,6 +59,8 @@ struct EncodeParams {
     int s_ld;                 // B side, fp32 scales: row length of the scale array
     int sf_blocks;            // UE8M0: number of 128-row blocks of the scale-tile array
     float amax_floor;
+    int b_tile;               // B side: 128 = one fp32 scale per 128 x 128 tile (blk 128 only), 0 = per column
+    int preround_bf16;        // B side: round each combination to bfloat16 before the maximum and the cast
 };
 
 struct CombParams {

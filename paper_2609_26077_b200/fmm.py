@@ -24,7 +24,8 @@ EXPORTS = ["fmm_plan_create", "fmm_plan_destroy", "fmm_workspace_bytes", "fmm_ma
 
 
 class QuantParams(C.Structure):
-    _fields_ = [("block_k", C.c_int), ("scale_mode", C.c_int), ("amax_floor", C.c_float), ("fp8_max", C.c_float)]
+    _fields_ = [("block_k", C.c_int), ("scale_mode", C.c_int), ("amax_floor", C.c_float), ("fp8_max", C.c_float),
+                ("b_tile_n", C.c_int), ("b_preround_bf16", C.c_int)]
 
 
 class FmmError(RuntimeError):
@@ -98,13 +99,14 @@ def _dev_ptr(t):
 class Plan:
     """fmm_plan_create / fmm_plan_destroy plus the calls that take a plan."""
 
-    def __init__(self, U=None, V=None, W=None, levels=1, block_k=32, scale_mode="fp32", amax_floor=1e-12):
+    def __init__(self, U=None, V=None, W=None, levels=1, block_k=32, scale_mode="fp32", amax_floor=1e-12,
+                 b_tile_n=0, b_preround_bf16=False):
         self.U, self.V, self.W = _coef(U), _coef(V), _coef(W)
         self.levels = int(levels)
         self.block_k = int(block_k)
         self.scale_mode = SCALE_MODES[scale_mode] if isinstance(scale_mode, str) else int(scale_mode)
         self.rank = 0 if self.U is None else int(self.U.shape[0])
-        qp = QuantParams(self.block_k, self.scale_mode, float(amax_floor), 448.0)
+        qp = QuantParams(self.block_k, self.scale_mode, float(amax_floor), 448.0, int(b_tile_n), int(bool(b_preround_bf16)))
         h = C.c_void_p()
         _check(lib().fmm_plan_create(C.byref(h), C.c_int(self.rank), _fptr(self.U), _fptr(self.V), _fptr(self.W),
                                      C.c_int(self.levels), C.byref(qp)), "fmm_plan_create")

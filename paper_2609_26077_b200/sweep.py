@@ -49,12 +49,16 @@ CONFIGS = {
                names=["cubic"] + P.LADDER, levels=[1]),
     # orbit-ratio stability (Table E.8): fifteen exact orbit members, one shape, signed-uniform operands
     "c8": dict(shape=(2048, 2048, 2048), families=["uniform"], trials=8, names=["cubic"] + P.ORBIT15, levels=[1]),
+    # weight-scale granularity (App. E.5): run with --block-k 128 and then again with --b-tile 128 [--b-bf16];
+    # heterogeneous synthetic weights stand in for the stored checkpoint tiles
+    "c9": dict(shape=(4096, 4096, 4096), families=["llm", "llm_hetero"], trials=8, names=ALL, levels=[1]),
     "c5": dict(shape=(2048, 2048, 2048), families=["scaled_gaussian", "student_t3"], trials=256, names=ALL, levels=[1, 2, 3]),
 }
 
 
 def _key(rec):
-    return (rec["config"], rec["family"], rec["seed"], rec["realization"], rec["levels"], rec["scale_mode"], rec["block_k"])
+    return (rec["config"], rec["family"], rec["seed"], rec["realization"], rec["levels"], rec["scale_mode"], rec["block_k"],
+            rec.get("b_tile", 0), rec.get("b_bf16", 0))
 
 
 def run(args):
@@ -75,9 +79,11 @@ def run(args):
         k = (name, lv)
         if k not in plans:
             if name == "cubic":
-                plans[k] = fmm.Plan(levels=0, block_k=args.block_k, scale_mode=args.scale_mode)
+                plans[k] = fmm.Plan(levels=0, block_k=args.block_k, scale_mode=args.scale_mode,
+                                    b_tile_n=args.b_tile, b_preround_bf16=args.b_bf16)
             else:
-                plans[k] = fmm.Plan(*P.get(name), levels=lv, block_k=args.block_k, scale_mode=args.scale_mode)
+                plans[k] = fmm.Plan(*P.get(name), levels=lv, block_k=args.block_k, scale_mode=args.scale_mode,
+                                    b_tile_n=args.b_tile, b_preround_bf16=args.b_bf16)
         return plans[k]
 
     out = open(args.out, "a")
@@ -86,7 +92,7 @@ def run(args):
     for family in cfg["families"]:
         for seed in range(trials):
             todo = [(n, lv) for n in cfg["names"] for lv in (cfg["levels"] if n != "cubic" else [0])
-                    if (args.config, family, seed, n, lv, args.scale_mode, args.block_k) not in done]
+                    if (args.config, family, seed, n, lv, args.scale_mode, args.block_k, args.b_tile, int(args.b_bf16)) not in done]
             if not todo:
                 continue
             A, B = Wl.FAMILIES[family](M, K, N, seed)
@@ -98,7 +104,8 @@ def run(args):
                 s = fmm.fmm_error_stats(C, ref).cpu().numpy()
                 st, code = pl.device_status()
                 rec = {"config": args.config, "family": family, "seed": seed, "realization": name, "levels": lv,
-                       "scale_mode": args.scale_mode, "block_k": args.block_k, "M": M, "K": K, "N": N,
+                       "scale_mode": args.scale_mode, "block_k": args.block_k, "b_tile": args.b_tile,
+                       "b_bf16": int(args.b_bf16), "M": M, "K": K, "N": N,
                        "sum_sq_diff": float(s[0]), "sum_sq_ref": float(s[1]), "max_abs_diff": float(s[2]),
                        "rel_frobenius": float(math.sqrt(s[0] / s[1])), "device_status": code}
                 out.write(json.dumps(rec) + "\n")
@@ -112,7 +119,8 @@ def summarise(path, file=sys.stdout):
     recs = [json.loads(line) for line in open(path) if line.strip()]
     groups = defaultdict(lambda: defaultdict(dict))
     for r in recs:
-        g = (r["config"], r["family"], r["scale_mode"], r["block_k"])
+        scales = r["scale_mode"] + ("+tile128" if r.get("b_tile") else "") + ("+bf16" if r.get("b_bf16") else "")
+        g = (r["config"], r["family"], scales, r["block_k"])
         groups[g][(r["realization"], r["levels"])][r["seed"]] = r
     rows = []
     for g, by in sorted(groups.items()):
@@ -185,6 +193,8 @@ def main():
     ap.add_argument("--config", choices=sorted(CONFIGS))
     ap.add_argument("--scale-mode", default="fp32", choices=["fp32", "ue8m0"])
     ap.add_argument("--block-k", type=int, default=32, choices=[32, 128])
+    ap.add_argument("--b-tile", type=int, default=0, choices=[0, 128], help="weight-side 128 x 128 scale tiles (blk 128, fp32)")
+    ap.add_argument("--b-bf16", action="store_true", help="bf16 pre-round of each encoded weight combination")
     ap.add_argument("--out", default="sweep.jsonl")
     ap.add_argument("--trials", type=int, default=0)
     ap.add_argument("--summarise")

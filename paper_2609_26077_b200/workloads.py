@@ -40,6 +40,17 @@ def llm_shaped(M, K, N, seed, outlier_sigma=1.5, weight_sigma=0.02):
     return A, B
 
 
+def llm_hetero_weights(M, K, N, seed, outlier_sigma=1.5, weight_sigma=0.02, col_sigma=1.0, row_sigma=0.5):
+    """As llm_shaped, with a weight matrix whose output channels (columns) and input channels (rows) carry
+    lognormal magnitude factors: the block-to-block heterogeneity that makes the weight-scale granularity
+    (one scale per column block vs per 128 x 128 tile, App. E.5) matter.  Stand-in for stored checkpoint
+    tiles, which are not available here."""
+    A, B = llm_shaped(M, K, N, seed, outlier_sigma, weight_sigma)
+    c = np.exp(np.float32(col_sigma) * _rng(seed, 3).standard_normal(N).astype(np.float32))
+    r = np.exp(np.float32(row_sigma) * _rng(seed, 4).standard_normal(K).astype(np.float32))
+    return A, (B * r[:, None] * c[None, :]).astype(np.float32)
+
+
 def log_uniform_sigma(seed, stream, lo=-3.0, hi=3.0):
     return float(10.0 ** _rng(seed, stream).uniform(lo, hi))
 
@@ -102,6 +113,7 @@ FAMILIES = {
     "gaussian": gaussian,
     "uniform": uniform,
     "llm": llm_shaped,
+    "llm_hetero": llm_hetero_weights,
     "scaled_gaussian": scaled_gaussian,
     "student_t3": student_t3,
     "rademacher": rademacher,
