@@ -164,9 +164,11 @@ def run_ours(args):
     C = torch.empty(M, N, device="cuda")
 
     def make_plan(name, levels, blk, mode):
+        # mode "fp32+tile128": fp32 scales with one weight-side scale per 128 x 128 tile (App. E.5)
+        kw = dict(block_k=blk, scale_mode=mode.split("+")[0], b_tile_n=128 if mode.endswith("+tile128") else 0)
         if name == "cubic" or levels == 0:
-            return fmm.Plan(levels=0, block_k=blk, scale_mode=mode)
-        return fmm.Plan(*P.get(name), levels=levels, block_k=blk, scale_mode=mode)
+            return fmm.Plan(levels=0, **kw)
+        return fmm.Plan(*P.get(name), levels=levels, **kw)
 
     def barrier():
         torch.cuda.synchronize()
@@ -287,6 +289,7 @@ def run_ours(args):
         todo = [("cubic", 0, args.block_k, args.scale_mode), ("strassen", 1, args.block_k, args.scale_mode),
                 ("phi_optimal", 1, 32, "ue8m0"), ("cubic", 0, 32, "ue8m0"),
                 ("phi_optimal", 1, 128, "fp32"), ("cubic", 0, 128, "fp32"), ("phi_optimal", 1, 32, "fp32"),
+                ("phi_optimal", 1, 128, "fp32+tile128"), ("cubic", 0, 128, "fp32+tile128"),
                 ("phi_optimal", 2, 32, "ue8m0")]
         seen = {(args.realization, args.levels, args.block_k, args.scale_mode)}
         for name, lv, blk, mode in todo:

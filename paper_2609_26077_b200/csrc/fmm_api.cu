@@ -182,6 +182,7 @@ fmm_status_t multiply(fmm_plan* plan, const FmmLayout& L, char* ws, float* C, in
     g.C = dest; g.ldc = pn; g.Mfull = parents * pm; g.Nfull = pn;
     g.m = (int)L.m; g.n = (int)L.n; g.k = (int)L.k; g.terms = (int)L.terms;
     g.out_start = plan->d_out_start; g.out = plan->d_out; g.status = plan->d_status;
+    g.sb_tile = plan->qp.b_tile_n == 128 ? 1 : 0;
     int launches = 0;
     fmm_status_t s = fmm_launch_gemm(g, plan->qp.block_k, (int)plan->qp.scale_mode, st, &launches);
     plan->last_launches += launches;

@@ -29,6 +29,11 @@
 namespace {
 using namespace fmmptx;
 
+// Internal third mode of the product kernel: FP32 scales whose B-side value is constant over each
+// 128-column tile (the 128 x 128 weight tiles of App. E.5).  The promotion then needs one multiply per row
+// and K block (s = sA * sB_tile) and one FMA per element, instead of a multiply and an FMA per element.
+constexpr int MODE_FP32_SB_TILE = 2;
+
 constexpr int BM = 128;                 // rows per CTA
 constexpr int BK = 128;                 // K elements (= bytes) per pipeline stage: one swizzle row
 constexpr int EPI_WARPS = 8;               // two per TMEM lane quadrant, each half of the tile's columns
@@ -411,12 +416,28 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                             for (int gi = 0; gi < C::GPB; ++gi) {
                                 const int g = g0 + gi;
                                 const ulonglong2* sbg = reinterpret_cast<const ulonglong2*>(sbs + (g * BN + h * C::CW) * 4);
-                                const unsigned long long sa2 = pack2(sa[g], sa[g]);
+                                float sab = sa[g];
+                                if (MODE == MODE_FP32_SB_TILE) sab *= *reinterpret_cast<const float*>(sbs + (g * BN + h * C::CW) * 4);
+                                const unsigned long long sa2 = pack2(sab, sab);
                                 const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (buf * C::GPB + gi) * BN + h * C::CW;
                                 uint32_t tmp[32];
 #pragma unroll
                                 for (int c = 0; c < C::CW / 32; ++c) {
                                     tmem_ld32(taddr + c * 32, tmp);      // a TMEM load round trip is a few tens of cycles
+                                    // the scale products do not depend on the accumulator: they are formed while the
+                                    // TMEM load is in flight (the wait below is a barrier for the compiler's scheduler)
+                                    // (measured: helps with one promotion per 128 k, hurts with one per 32 k, where the
+                                    // compiler's own interleaving of the two granules is better)
+                                    constexpr bool HOIST = (BLK == 128) && MODE != MODE_FP32_SB_TILE;
+                                    unsigned long long sp[HOIST ? 16 : 1];
+                                    if (HOIST) {
+#pragma unroll
+                                        for (int i = 0; i < 8; ++i) {
+                                            const ulonglong2 s4 = sbg[c * 8 + i];        // four column scales
+                                            sp[HOIST ? 2 * i : 0] = mul2(sa2, s4.x);
+                                            sp[HOIST ? 2 * i + 1 : 0] = mul2(sa2, s4.y);
+                                        }
+                                    }
                                     tmem_ld_wait();
                                     if (gi + 1 == C::GPB && c + 1 == C::CW / 32) {
                                         // the last chunk is in registers: hand the TMEM buffers back before the arithmetic
@@ -426,10 +447,15 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                                     }
 #pragma unroll
                                     for (int i = 0; i < 8; ++i) {
-                                        const ulonglong2 s4 = sbg[c * 8 + i];        // four column scales
                                         const uint32_t* tp = tmp + 4 * i;
-                                        acc2[c * 16 + 2 * i] = fma2(pack2u(tp[0], tp[1]), mul2(sa2, s4.x), acc2[c * 16 + 2 * i]);
-                                        acc2[c * 16 + 2 * i + 1] = fma2(pack2u(tp[2], tp[3]), mul2(sa2, s4.y), acc2[c * 16 + 2 * i + 1]);
+                                        unsigned long long s01 = sa2, s23 = sa2;        // tile mode: sA * sB_tile
+                                        if (HOIST) { s01 = sp[HOIST ? 2 * i : 0]; s23 = sp[HOIST ? 2 * i + 1 : 0]; }
+                                        else if (MODE != MODE_FP32_SB_TILE) {
+                                            const ulonglong2 s4 = sbg[c * 8 + i];        // four column scales
+                                            s01 = mul2(sa2, s4.x); s23 = mul2(sa2, s4.y);
+                                        }
+                                        acc2[c * 16 + 2 * i] = fma2(pack2u(tp[0], tp[1]), s01, acc2[c * 16 + 2 * i]);
+                                        acc2[c * 16 + 2 * i + 1] = fma2(pack2u(tp[2], tp[3]), s23, acc2[c * 16 + 2 * i + 1]);
                                     }
                                 }
                             }
@@ -615,6 +641,11 @@ fmm_status_t launch_shape(const GemmParams& g, cudaStream_t st)
     // on the CUDA cores and use 128-column tiles, whose four TMEM accumulators let the MMA issuer run
     // further ahead of the promoting warps.
     if constexpr (MODE != FMM_SCALE_UE8M0_CEIL) {
+        if constexpr (BLK == 128) {
+            // one promotion per 128 k: the tensor pipe matters again, and 256-column instructions read half as
+            // much shared memory per flop as 128-column ones
+            if ((g.m % 256) == 0 && (g.n % 256) == 0) return launch<256, MODE, BLK, 2>(g, st);
+        }
         if ((g.m % 256) == 0) return launch<128, MODE, BLK, 2>(g, st);
         return launch<128, MODE, BLK, 1>(g, st);
     } else {
@@ -636,6 +667,7 @@ fmm_status_t fmm_launch_gemm(const GemmParams& g, int blk, int mode, cudaStream_
 {
     fmm_status_t s;
     if (mode == FMM_SCALE_UE8M0_CEIL) s = launch_shape<FMM_SCALE_UE8M0_CEIL, 32>(g, st);
+    else if (blk == 128 && g.sb_tile) s = launch_shape<MODE_FP32_SB_TILE, 128>(g, st);
     else if (blk == 32) s = launch_shape<FMM_SCALE_FP32_AMAX_DIV_448, 32>(g, st);
     else s = launch_shape<FMM_SCALE_FP32_AMAX_DIV_448, 128>(g, st);
     if (s == FMM_OK && launches) *launches += 1;

@@ -92,6 +92,7 @@ struct GemmParams {
     int m, n, k, terms;
     const int* out_start; const FmmOutEntry* out;
     int* status;
+    int sb_tile;                            // fp32 scales, blk 128: the B-side scale is constant over each 128-column tile
 };
 fmm_status_t fmm_launch_bounded_wait_selftest(int* status, unsigned long long limit_ns, cudaStream_t st);
 fmm_status_t fmm_launch_gemm(const GemmParams& p, int blk, int mode, cudaStream_t st, int* launches);
