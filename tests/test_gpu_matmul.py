@@ -38,6 +38,7 @@ CASES = [
     ("winograd_rb", 2, (512, 512, 512), 32, "ue8m0", "gaussian"),
     ("strassen", 1, (5120, 512, 4096), 32, "ue8m0", "gaussian"),
     ("phi_optimal", 1, (4864, 256, 4096), 32, "ue8m0", "uniform"),
+    ("strassen", 1, (5120, 512, 4096), 128, "fp32", "gaussian"),
 ]
 
 
