@@ -137,7 +137,10 @@ fmm_status_t encode_side(fmm_plan* plan, const FmmLayout& L, char* ws, const flo
         const float* cur = X;
         int64_t cur_rows = rows, cur_cols = cols, cur_ld = cols, cur_stride = 0;
         int batch = 1;
-        for (int level = 1; level < lv; ++level) {
+        // the last two levels run as one kernel where that is supported: the combinations of level lv-1 stay
+        // in registers
+        const bool fused2 = lv >= 2 && fmm_encode2_supported(b_side, blk, e.b_tile, e.preround_bf16);
+        for (int level = 1; level < (fused2 ? lv - 1 : lv); ++level) {
             CombParams c;
             memset(&c, 0, sizeof(c));
             c.in = cur; c.in_batch_stride = cur_stride; c.ld = cur_ld; c.batch = batch;
@@ -151,10 +154,17 @@ fmm_status_t encode_side(fmm_plan* plan, const FmmLayout& L, char* ws, const flo
             batch *= R;
         }
         e.in = cur; e.in_batch_stride = cur_stride; e.ld = cur_ld; e.batch = batch;
-        e.rows = (int)(cur_rows / 2); e.cols = (int)(cur_cols / 2); e.nq = 4; e.R = R;
+        const int div = fused2 ? 4 : 2;
+        e.rows = (int)(cur_rows / div); e.cols = (int)(cur_cols / div); e.nq = 4; e.R = R;
         e.qoff[0] = 0; e.qoff[1] = e.cols; e.qoff[2] = (int64_t)e.rows * e.ld; e.qoff[3] = (int64_t)e.rows * e.ld + e.cols;
+        for (int j = 0; j < 4; ++j) e.qoff_outer[j] = 2 * e.qoff[j];
         fill_coef(e.coef, coef, R);
         e.s_step = 0; e.s_ld = e.cols; e.sf_blocks = (b_side ? e.cols : e.rows) / 128;
+        if (fused2) {
+            s = b_side ? fmm_launch_encode2_b(e, mode, st) : fmm_launch_encode2_a(e, blk, mode, st);
+            if (s == FMM_OK) plan->last_launches++;
+            return s;
+        }
     }
     s = b_side ? fmm_launch_encode_b(e, blk, mode, st) : fmm_launch_encode_a(e, blk, mode, st);
     if (s == FMM_OK) plan->last_launches++;

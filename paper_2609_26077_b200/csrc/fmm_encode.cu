@@ -76,6 +76,126 @@ template <uint32_t NZ> __device__ __forceinline__ bool coef_used(int r, int j, f
 template <uint32_t NZ> __device__ __forceinline__ bool row_used(int r, int R)
 { return NZ ? ((NZ >> (4 * r)) & 15u) != 0 : (r < R); }
 
+// The arithmetic of one chunk, shared by the one-level and two-level kernels.  x[j] holds four consecutive
+// elements (along the contracted axis) of input block j; the GROUP lanes that share a quantization block are
+// adjacent.  Forms the R combinations v[r], reduces their block maxima with a transposing butterfly over the
+// 8 lanes (lane & 7) - afterwards each lane holds the maximum of combination (lane & 7) - and computes that
+// combination's multiplier `inv` and stored scale (s or e8) once per block instead of once per lane.
+template <int GROUP, int MODE, uint32_t NZ>
+__device__ __forceinline__ void combine_chunk(const EncodeParams& p, const float4 (&x)[4], int lane,
+                                              float4 (&v)[FMM_MAX_RANK], float& inv, float& s, uint32_t& e8)
+{
+    constexpr unsigned FULL = 0xffffffffu;
+    const bool b2 = lane & 4, b1 = lane & 2, b0 = lane & 1;
+    float am[FMM_MAX_RANK];
+#pragma unroll
+    for (int r = 0; r < FMM_MAX_RANK; ++r) {
+        v[r] = make_float4(0.f, 0.f, 0.f, 0.f); am[r] = 0.0f;
+        if (row_used<NZ>(r, p.R)) {
+            bool set = false;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const float cj = p.coef[r][j];
+                if (coef_used<NZ>(r, j, cj)) {
+                    if (!set) {
+                        v[r].x = __fmul_rn(cj, x[j].x); v[r].y = __fmul_rn(cj, x[j].y);
+                        v[r].z = __fmul_rn(cj, x[j].z); v[r].w = __fmul_rn(cj, x[j].w);
+                        set = true;
+                    } else {
+                        v[r].x = __fmaf_rn(cj, x[j].x, v[r].x); v[r].y = __fmaf_rn(cj, x[j].y, v[r].y);
+                        v[r].z = __fmaf_rn(cj, x[j].z, v[r].z); v[r].w = __fmaf_rn(cj, x[j].w, v[r].w);
+                    }
+                }
+            }
+            am[r] = fmaxf(fmaxf(fabsf(v[r].x), fabsf(v[r].y)), fmaxf(fabsf(v[r].z), fabsf(v[r].w)));
+        }
+    }
+    float w[4], x2[2], mine;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const float send = b2 ? am[j] : am[j + 4], keep = b2 ? am[j + 4] : am[j];
+        w[j] = fmaxf(keep, __shfl_xor_sync(FULL, send, 4));
+    }
+#pragma unroll
+    for (int j = 0; j < 2; ++j) {
+        const float send = b1 ? w[j] : w[j + 2], keep = b1 ? w[j + 2] : w[j];
+        x2[j] = fmaxf(keep, __shfl_xor_sync(FULL, send, 2));
+    }
+    {
+        const float send = b0 ? x2[0] : x2[1], keep = b0 ? x2[1] : x2[0];
+        mine = fmaxf(keep, __shfl_xor_sync(FULL, send, 1));
+    }
+    if (GROUP == 32) {
+        mine = fmaxf(mine, __shfl_xor_sync(FULL, mine, 8));
+        mine = fmaxf(mine, __shfl_xor_sync(FULL, mine, 16));
+    }
+    inv = block_scale<MODE>(mine, p.amax_floor, s, e8);
+}
+
+// One combination of the outer level, in registers: the same rounded-multiply / FMA chain as above.
+template <uint32_t NZ>
+__device__ __forceinline__ float4 combine_outer(const EncodeParams& p, int r, const float4 (&raw)[4][4], int q2)
+{
+    float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
+    bool set = false;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const float cj = p.coef[r][j];
+        if (coef_used<NZ>(r, j, cj)) {
+            const float4 a = raw[j][q2];
+            if (!set) {
+                o.x = __fmul_rn(cj, a.x); o.y = __fmul_rn(cj, a.y); o.z = __fmul_rn(cj, a.z); o.w = __fmul_rn(cj, a.w);
+                set = true;
+            } else {
+                o.x = __fmaf_rn(cj, a.x, o.x); o.y = __fmaf_rn(cj, a.y, o.y);
+                o.z = __fmaf_rn(cj, a.z, o.z); o.w = __fmaf_rn(cj, a.w, o.w);
+            }
+        }
+    }
+    return o;
+}
+
+// A-side stores of one chunk: four code bytes per lane and combination; the scale of combination (lane & 7).
+// b = index of the input matrix (terms b*R .. b*R + R-1), i = leaf row, c = 128-k chunk.
+template <int BLK, int MODE, uint32_t NZ>
+__device__ __forceinline__ void store_chunk_a(const EncodeParams& p, const float4 (&v)[FMM_MAX_RANK], float inv, float s,
+                                              uint32_t e8, int b, int i, int c, int lane)
+{
+    constexpr int GROUP = BLK / 4;
+    constexpr unsigned FULL = 0xffffffffu;
+    const int64_t term_codes = (int64_t)p.rows * p.cols;
+    const int nkb = p.cols / BLK;
+    const int my_r = lane & 7;
+    uint8_t* qp = p.q_out + ((int64_t)b * p.R) * term_codes + (int64_t)i * p.cols + c * 128 + lane * 4;
+#pragma unroll
+    for (int r = 0; r < FMM_MAX_RANK; ++r) {
+        if (row_used<NZ>(r, p.R)) {
+            const float inv_r = __shfl_sync(FULL, inv, (GROUP == 32) ? r : ((lane & 24) | r));
+            *reinterpret_cast<uint32_t*>(qp) = pack4_e4m3(__fmul_rn(v[r].x, inv_r), __fmul_rn(v[r].y, inv_r),
+                                                          __fmul_rn(v[r].z, inv_r), __fmul_rn(v[r].w, inv_r));
+        }
+        qp += term_codes;
+    }
+    // scales: lane holds the scale of combination my_r, block (lane / GROUP) of this chunk
+    if (MODE == FMM_SCALE_FP32_AMAX_DIV_448) {
+        if (my_r < p.R && (GROUP == 8 || lane < 8)) {
+            float* so = reinterpret_cast<float*>(reinterpret_cast<char*>(p.s_out) + ((int64_t)b * p.R + my_r) * p.s_term_stride);
+            so[(int64_t)i * nkb + c * (128 / BLK) + (GROUP == 8 ? (lane >> 3) : 0)] = s;
+        }
+    } else {
+        // four exponent bytes of this row (blocks 4c .. 4c+3) form one aligned word of the scale tile
+        uint32_t wv = e8 << (8 * (lane >> 3));
+        wv |= __shfl_xor_sync(FULL, wv, 8);
+        wv |= __shfl_xor_sync(FULL, wv, 16);
+        if (lane < 8 && lane < p.R) {
+            char* so = reinterpret_cast<char*>(p.s_out) + ((int64_t)b * p.R + lane) * p.s_term_stride;
+            const int ig = i + lane * p.s_step;            // row inside the scale-tile array
+            const int64_t tile = (int64_t)c * p.sf_blocks + (ig >> 7);
+            *reinterpret_cast<uint32_t*>(so + tile * 512 + (ig & 31) * 16 + ((ig & 127) >> 5) * 4) = wv;
+        }
+    }
+}
+
 template <int BLK, int MODE, uint32_t NZ>
 __global__ void __launch_bounds__(256) encode_a_kernel(const EncodeParams p)
 {
@@ -85,15 +205,11 @@ __global__ void __launch_bounds__(256) encode_a_kernel(const EncodeParams p)
     const uint32_t warp_gid = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const uint32_t nwarps = (gridDim.x * blockDim.x) >> 5;
     const int chunks = p.cols / 128;
-    const int nkb = p.cols / BLK;
     // a task is CPT consecutive 128-k chunks of one output row; tasks are dealt to warps round-robin
     // (32-bit index arithmetic only: one division per task, none per chunk)
     const int CPT = (chunks % 8 == 0) ? 8 : ((chunks % 4 == 0) ? 4 : 1);
     const uint32_t tasks_per_row = (uint32_t)(chunks / CPT);
     const uint32_t tasks = (uint32_t)p.batch * (uint32_t)p.rows * tasks_per_row;
-    const int64_t term_codes = (int64_t)p.rows * p.cols;
-    const bool b2 = lane & 4, b1 = lane & 2, b0 = lane & 1;
-    const int my_r = lane & 7;
 
     for (uint32_t task = warp_gid; task < tasks; task += nwarps) {
       const uint32_t row_id = task / tasks_per_row;
@@ -117,81 +233,10 @@ __global__ void __launch_bounds__(256) encode_a_kernel(const EncodeParams p)
         }
 
         float4 v[FMM_MAX_RANK];
-        float am[FMM_MAX_RANK];
-#pragma unroll
-        for (int r = 0; r < FMM_MAX_RANK; ++r) {
-            v[r] = make_float4(0.f, 0.f, 0.f, 0.f); am[r] = 0.0f;
-            if (row_used<NZ>(r, p.R)) {
-                bool set = false;
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const float cj = p.coef[r][j];
-                    if (coef_used<NZ>(r, j, cj)) {
-                        if (!set) {
-                            v[r].x = __fmul_rn(cj, x[j].x); v[r].y = __fmul_rn(cj, x[j].y);
-                            v[r].z = __fmul_rn(cj, x[j].z); v[r].w = __fmul_rn(cj, x[j].w);
-                            set = true;
-                        } else {
-                            v[r].x = __fmaf_rn(cj, x[j].x, v[r].x); v[r].y = __fmaf_rn(cj, x[j].y, v[r].y);
-                            v[r].z = __fmaf_rn(cj, x[j].z, v[r].z); v[r].w = __fmaf_rn(cj, x[j].w, v[r].w);
-                        }
-                    }
-                }
-                am[r] = fmaxf(fmaxf(fabsf(v[r].x), fabsf(v[r].y)), fmaxf(fabsf(v[r].z), fabsf(v[r].w)));
-            }
-        }
-        // transposing butterfly over the 8 lanes (lane & 7): afterwards `mine` is the maximum of
-        // combination (lane & 7) over those lanes
-        float w[4], x2[2], mine;
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const float send = b2 ? am[j] : am[j + 4], keep = b2 ? am[j + 4] : am[j];
-            w[j] = fmaxf(keep, __shfl_xor_sync(FULL, send, 4));
-        }
-#pragma unroll
-        for (int j = 0; j < 2; ++j) {
-            const float send = b1 ? w[j] : w[j + 2], keep = b1 ? w[j + 2] : w[j];
-            x2[j] = fmaxf(keep, __shfl_xor_sync(FULL, send, 2));
-        }
-        {
-            const float send = b0 ? x2[0] : x2[1], keep = b0 ? x2[1] : x2[0];
-            mine = fmaxf(keep, __shfl_xor_sync(FULL, send, 1));
-        }
-        if (GROUP == 32) {
-            mine = fmaxf(mine, __shfl_xor_sync(FULL, mine, 8));
-            mine = fmaxf(mine, __shfl_xor_sync(FULL, mine, 16));
-        }
-        float s; uint32_t e8;
-        const float inv = block_scale<MODE>(mine, p.amax_floor, s, e8);
+        float inv, s; uint32_t e8;
+        combine_chunk<GROUP, MODE, NZ>(p, x, lane, v, inv, s, e8);
 
-        uint8_t* qp = p.q_out + ((int64_t)b * p.R) * term_codes + (int64_t)i * p.cols + c * 128 + lane * 4;
-#pragma unroll
-        for (int r = 0; r < FMM_MAX_RANK; ++r) {
-            if (row_used<NZ>(r, p.R)) {
-                const float inv_r = __shfl_sync(FULL, inv, (GROUP == 32) ? r : ((lane & 24) | r));
-                *reinterpret_cast<uint32_t*>(qp) = pack4_e4m3(__fmul_rn(v[r].x, inv_r), __fmul_rn(v[r].y, inv_r),
-                                                              __fmul_rn(v[r].z, inv_r), __fmul_rn(v[r].w, inv_r));
-            }
-            qp += term_codes;
-        }
-        // scales: lane holds the scale of combination my_r, block (lane / GROUP) of this chunk
-        if (MODE == FMM_SCALE_FP32_AMAX_DIV_448) {
-            if (my_r < p.R && (GROUP == 8 || lane < 8)) {
-                float* so = reinterpret_cast<float*>(reinterpret_cast<char*>(p.s_out) + ((int64_t)b * p.R + my_r) * p.s_term_stride);
-                so[(int64_t)i * nkb + c * (128 / BLK) + (GROUP == 8 ? (lane >> 3) : 0)] = s;
-            }
-        } else {
-            // four exponent bytes of this row (blocks 4c .. 4c+3) form one aligned word of the scale tile
-            uint32_t wv = e8 << (8 * (lane >> 3));
-            wv |= __shfl_xor_sync(FULL, wv, 8);
-            wv |= __shfl_xor_sync(FULL, wv, 16);
-            if (lane < 8 && lane < p.R) {
-                char* so = reinterpret_cast<char*>(p.s_out) + ((int64_t)b * p.R + lane) * p.s_term_stride;
-                const int ig = i + lane * p.s_step;            // row inside the scale-tile array
-                const int64_t tile = (int64_t)c * p.sf_blocks + (ig >> 7);
-                *reinterpret_cast<uint32_t*>(so + tile * 512 + (ig & 31) * 16 + ((ig & 127) >> 5) * 4) = wv;
-            }
-        }
+        store_chunk_a<BLK, MODE, NZ>(p, v, inv, s, e8, b, i, c, lane);
       }
     }
 }
@@ -338,7 +383,108 @@ __global__ void __launch_bounds__(TILE ? 256 : 128, TILE ? 2 : 4) encode_b_kerne
     }
 }
 
-// fp32 combinations of the outer recursion levels (levels >= 2): out[b*R + r] = sum_j coef[r][j] X_j
+// ---------------------------------------------------------------------------------------------
+// Two recursion levels in one pass (levels >= 2): the combinations of the second-to-last level are formed in
+// registers from the 16 sub-blocks and fed to the leaf-level arithmetic above, so the 7 fp32 intermediate
+// matrices of that level are neither written nor read back.  The rounding sequence is the one of the
+// level-by-level evaluation (Sec. 3: recursion = Kronecker power; each level a rounded multiply / FMA chain
+// in fp32), so the bytes are identical.  p.rows x p.cols are the leaf dimensions, the input matrices are
+// 4*rows x 4*cols, p.qoff_outer[] / p.qoff[] the block offsets of the two levels; terms are numbered
+// (b * R + r1) * R + r2.
+template <int BLK, int MODE, uint32_t NZ>
+__global__ void __launch_bounds__(256) encode2_a_kernel(const EncodeParams p)
+{
+    constexpr int GROUP = BLK / 4;
+    const int lane = threadIdx.x & 31;
+    const uint32_t warp_gid = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const uint32_t nwarps = (gridDim.x * blockDim.x) >> 5;
+    const uint32_t chunks = (uint32_t)(p.cols / 128);
+    const uint32_t tasks = (uint32_t)p.batch * (uint32_t)p.rows * chunks;       // one 128-k chunk of one leaf row
+    for (uint32_t task = warp_gid; task < tasks; task += nwarps) {
+        const uint32_t row_id = task / chunks;
+        const int c = (int)(task - row_id * chunks);
+        const int b = (int)(row_id / (uint32_t)p.rows);
+        const int i = (int)(row_id - (uint32_t)b * (uint32_t)p.rows);
+        const float* base = p.in + (int64_t)b * p.in_batch_stride + (int64_t)i * p.ld + c * 128 + lane * 4;
+        float4 raw[4][4];                                   // [outer block][inner block]
+#pragma unroll
+        for (int q1 = 0; q1 < 4; ++q1)
+#pragma unroll
+            for (int q2 = 0; q2 < 4; ++q2)
+                raw[q1][q2] = __ldcs(reinterpret_cast<const float4*>(base + p.qoff_outer[q1] + p.qoff[q2]));
+#pragma unroll
+        for (int r1 = 0; r1 < FMM_MAX_RANK; ++r1) {
+            if (row_used<NZ>(r1, p.R)) {
+                float4 x[4];
+#pragma unroll
+                for (int q2 = 0; q2 < 4; ++q2) x[q2] = combine_outer<NZ>(p, r1, raw, q2);
+                float4 v[FMM_MAX_RANK];
+                float inv, s; uint32_t e8;
+                combine_chunk<GROUP, MODE, NZ>(p, x, lane, v, inv, s, e8);
+                store_chunk_a<BLK, MODE, NZ>(p, v, inv, s, e8, b * p.R + r1, i, c, lane);
+            }
+        }
+    }
+}
+
+// B side, block 32: a thread owns 4 consecutive k of one column, the 8 lanes (lane & 7) of a column hold one
+// 32-element block, a warp covers 4 adjacent columns (16-byte row segments; the neighbouring warp of the block
+// uses the other half of each 32-byte sector).  The eight lanes of a column write 32 contiguous code bytes of
+// the K-major output.  Grid: (cols / 32, rows / 32, batch), 256 threads.
+template <int MODE, uint32_t NZ>
+__global__ void __launch_bounds__(256) encode2_b_kernel(const EncodeParams p)
+{
+    constexpr unsigned FULL = 0xffffffffu;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int j = blockIdx.x * 32 + warp * 4 + (lane >> 3);        // leaf column
+    const int kb = blockIdx.y;                                      // 32-k block
+    const int k0 = kb * 32 + (lane & 7) * 4;
+    const int b = blockIdx.z;
+    const float* base = p.in + (int64_t)b * p.in_batch_stride + (int64_t)k0 * p.ld + j;
+    const int64_t term_codes = (int64_t)p.rows * p.cols;
+    const int my_r = lane & 7;
+    float4 raw[4][4];
+#pragma unroll
+    for (int q1 = 0; q1 < 4; ++q1)
+#pragma unroll
+        for (int q2 = 0; q2 < 4; ++q2) {
+            const float* src = base + p.qoff_outer[q1] + p.qoff[q2];
+            raw[q1][q2] = make_float4(__ldg(src), __ldg(src + p.ld), __ldg(src + 2 * p.ld), __ldg(src + 3 * p.ld));
+        }
+#pragma unroll
+    for (int r1 = 0; r1 < FMM_MAX_RANK; ++r1) {
+        if (row_used<NZ>(r1, p.R)) {
+            float4 x[4];
+#pragma unroll
+            for (int q2 = 0; q2 < 4; ++q2) x[q2] = combine_outer<NZ>(p, r1, raw, q2);
+            float4 v[FMM_MAX_RANK];
+            float inv, s; uint32_t e8;
+            combine_chunk<8, MODE, NZ>(p, x, lane, v, inv, s, e8);
+            const int64_t t0 = ((int64_t)b * p.R + r1) * p.R;
+            uint8_t* qp = p.q_out + t0 * term_codes + (int64_t)j * p.rows + k0;
+#pragma unroll
+            for (int r = 0; r < FMM_MAX_RANK; ++r) {
+                if (row_used<NZ>(r, p.R)) {
+                    const float inv_r = __shfl_sync(FULL, inv, (lane & 24) | r);
+                    *reinterpret_cast<uint32_t*>(qp) = pack4_e4m3(__fmul_rn(v[r].x, inv_r), __fmul_rn(v[r].y, inv_r),
+                                                                  __fmul_rn(v[r].z, inv_r), __fmul_rn(v[r].w, inv_r));
+                }
+                qp += term_codes;
+            }
+            if (my_r < p.R) {
+                char* so = reinterpret_cast<char*>(p.s_out) + (t0 + my_r) * p.s_term_stride;
+                if (MODE == FMM_SCALE_FP32_AMAX_DIV_448) {
+                    reinterpret_cast<float*>(so)[(int64_t)kb * p.s_ld + j] = s;
+                } else {
+                    const int64_t tile = (int64_t)(kb >> 2) * p.sf_blocks + (j >> 7);
+                    *reinterpret_cast<uint8_t*>(so + tile * 512 + (j & 31) * 16 + ((j & 127) >> 5) * 4 + (kb & 3)) = (uint8_t)e8;
+                }
+            }
+        }
+    }
+}
+
+// fp32 combinations of the outer recursion levels (levels >= 3): out[b*R + r] = sum_j coef[r][j] X_j
 __global__ void __launch_bounds__(256) comb_kernel(const CombParams p)
 {
     const int c4 = p.cols / 4;
@@ -489,6 +635,26 @@ void launch_b(const EncodeParams& p, dim3 grid, cudaStream_t st)
         default: encode_b_kernel<BLK, MODE, 0u, false, false><<<grid, 128, 0, st>>>(p); return;
     }
 }
+template <int BLK, int MODE>
+void launch_a2(const EncodeParams& p, unsigned g, cudaStream_t st)
+{
+    switch (coef_mask(p)) {
+#define X(M) case M: encode2_a_kernel<BLK, MODE, M><<<g, 256, 0, st>>>(p); return;
+        FMM_KNOWN_MASKS(X)
+#undef X
+        default: encode2_a_kernel<BLK, MODE, 0u><<<g, 256, 0, st>>>(p); return;
+    }
+}
+template <int MODE>
+void launch_b2(const EncodeParams& p, dim3 grid, cudaStream_t st)
+{
+    switch (coef_mask(p)) {
+#define X(M) case M: encode2_b_kernel<MODE, M><<<grid, 256, 0, st>>>(p); return;
+        FMM_KNOWN_MASKS(X)
+#undef X
+        default: encode2_b_kernel<MODE, 0u><<<grid, 256, 0, st>>>(p); return;
+    }
+}
 // weight-side options (tile scales and / or bf16 pre-round): blk 128, fp32 scales
 template <bool TILE, bool PRE>
 void launch_b_opt(const EncodeParams& p, dim3 grid, cudaStream_t st)
@@ -537,5 +703,36 @@ fmm_status_t fmm_launch_encode_b(const EncodeParams& p, int blk, int mode, cudaS
     } else {
         launch_b<32, FMM_SCALE_UE8M0_CEIL>(p, grid, st);
     }
+    return cudaGetLastError() == cudaSuccess ? FMM_OK : FMM_ERR_CUDA;
+}
+
+bool fmm_encode2_supported(bool b_side, int blk, int b_tile, int preround_bf16)
+{
+    // A side: every block size; B side: block 32 (a 128-element block along the strided axis would leave one
+    // column per warp), no weight-side options
+    return !b_side || (blk == 32 && !b_tile && !preround_bf16);
+}
+
+fmm_status_t fmm_launch_encode2_a(const EncodeParams& p, int blk, int mode, cudaStream_t st)
+{
+    const int64_t tasks = (int64_t)p.batch * p.rows * (p.cols / 128);
+    int64_t blocks = (tasks + 7) / 8;
+    const int64_t cap = (int64_t)sm_count() * 64;
+    if (blocks > cap) blocks = cap;
+    const unsigned g = (unsigned)blocks;
+    if (mode == FMM_SCALE_FP32_AMAX_DIV_448) {
+        if (blk == 32) launch_a2<32, FMM_SCALE_FP32_AMAX_DIV_448>(p, g, st);
+        else launch_a2<128, FMM_SCALE_FP32_AMAX_DIV_448>(p, g, st);
+    } else {
+        launch_a2<32, FMM_SCALE_UE8M0_CEIL>(p, g, st);
+    }
+    return cudaGetLastError() == cudaSuccess ? FMM_OK : FMM_ERR_CUDA;
+}
+
+fmm_status_t fmm_launch_encode2_b(const EncodeParams& p, int mode, cudaStream_t st)
+{
+    dim3 grid((unsigned)(p.cols / 32), (unsigned)(p.rows / 32), (unsigned)p.batch);
+    if (mode == FMM_SCALE_FP32_AMAX_DIV_448) launch_b2<FMM_SCALE_FP32_AMAX_DIV_448>(p, grid, st);
+    else launch_b2<FMM_SCALE_UE8M0_CEIL>(p, grid, st);
     return cudaGetLastError() == cudaSuccess ? FMM_OK : FMM_ERR_CUDA;
 }

@@ -49,6 +49,7 @@ struct EncodeParams {
     int batch;                // number of input matrices
     int rows, cols;           // leaf (output) dimensions per combination
     int64_t qoff[4];          // element offsets of the four input blocks that are combined
+    int64_t qoff_outer[4];    // two-level kernels: offsets of the four blocks of the outer level
     int nq;                   // number of input blocks read (4, or 1 for a plain pass over one matrix)
     int R;                    // combinations per input matrix
     float coef[FMM_MAX_RANK][4];
@@ -82,6 +83,10 @@ fmm_status_t fmm_launch_decode(const DecodeParams& p, cudaStream_t st);
 fmm_status_t fmm_launch_comb(const CombParams& p, cudaStream_t st);
 fmm_status_t fmm_launch_encode_a(const EncodeParams& p, int blk, int mode, cudaStream_t st);
 fmm_status_t fmm_launch_encode_b(const EncodeParams& p, int blk, int mode, cudaStream_t st);
+// last two recursion levels in one pass (p.rows x p.cols = leaf dimensions, inputs 4*rows x 4*cols)
+bool fmm_encode2_supported(bool b_side, int blk, int b_tile, int preround_bf16);
+fmm_status_t fmm_launch_encode2_a(const EncodeParams& p, int blk, int mode, cudaStream_t st);
+fmm_status_t fmm_launch_encode2_b(const EncodeParams& p, int mode, cudaStream_t st);
 
 struct GemmParams {
     const uint8_t* qa; const uint8_t* qb;   // terms x m x k, terms x n x k

@@ -25,6 +25,15 @@ CASES = [
     ("cubic8", 1, (256, 256, 256), 32, "fp32", "gaussian"),
     ("phi_optimal", 1, (256, 256, 256), 32, "fp32", "scaled_gaussian"),
     ("strassen", 1, (256, 256, 256), 128, "fp32", "student_t3"),
+    # last two recursion levels in one kernel: rectangular shapes, every scale mode, a realization without a
+    # pre-instantiated zero pattern, block 128 (two-level kernel on the A side only), three levels
+    ("phi_optimal", 2, (512, 1536, 1024), 32, "fp32", "llm"),
+    ("winograd", 2, (1024, 512, 1536), 32, "ue8m0", "student_t3"),
+    ("pert_f1_diag_m_rb", 2, (512, 512, 1024), 32, "ue8m0", "gaussian"),
+    ("pert_f2_shear_p_rb", 2, (512, 1024, 512), 32, "fp32", "uniform"),
+    ("phi_optimal", 2, (512, 1024, 512), 128, "fp32", "gaussian"),
+    ("cubic8", 2, (512, 512, 512), 32, "ue8m0", "gaussian"),
+    ("phi_optimal", 3, (1024, 1024, 2048), 32, "ue8m0", "scaled_gaussian"),
 ]
 
 
