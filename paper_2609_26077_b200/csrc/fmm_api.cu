@@ -191,6 +191,7 @@ fmm_status_t multiply(fmm_plan* plan, const FmmLayout& L, char* ws, float* C, in
     float* dest = lv >= 2 ? reinterpret_cast<float*>(ws + L.dec[lv - 1]) : C;
     g.C = dest; g.ldc = pn; g.Mfull = parents * pm; g.Nfull = pn;
     g.m = (int)L.m; g.n = (int)L.n; g.k = (int)L.k; g.terms = (int)L.terms;
+    g.terms_per_group = plan->levels >= 2 ? plan->rank : (int)L.terms;
     g.out_start = plan->d_out_start; g.out = plan->d_out; g.status = plan->d_status;
     g.sb_tile = plan->qp.b_tile_n == 128 ? 1 : 0;
     int launches = 0;

@@ -150,7 +150,10 @@ struct KParams {
     const uint8_t* sa; const uint8_t* sb;   // scale arrays (bytes); fp32 mode only
     long long sa_term, sb_term;
     int m, n, k, terms;
-    int split_from, items;                  // positions >= split_from are cut into two 128-column items
+    // Work items.  A slot is (term group, tile position): the terms of one group (the R products of one parent
+    // at the innermost level; all terms at one level) feed one set of output blocks and are walked by one CTA
+    // (pair) in order.  Slots >= split_from are cut into two 128-column items.
+    int positions, terms_per_group, split_from, items;
     const int* out_start; const FmmOutEntry* out;
     int* status;
 };
@@ -208,7 +211,7 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
 
     const int tiles_n = p.n / BN;
     // work item w -> tile position, column offset inside the position, half-width flag
-    auto item_pos = [&](int w) { return (C::SPLIT && w >= p.split_from) ? p.split_from + ((w - p.split_from) >> 1) : w; };
+    auto item_slot = [&](int w) { return (C::SPLIT && w >= p.split_from) ? p.split_from + ((w - p.split_from) >> 1) : w; };
     auto item_half = [&](int w) { return C::SPLIT && w >= p.split_from; };
     auto item_coff = [&](int w) { return (C::SPLIT && w >= p.split_from) ? ((w - p.split_from) & 1) * (BN / 2) : 0; };
     const int kstages = p.k / BK;
@@ -224,11 +227,12 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             int ss = 0; uint32_t sphase = 0;
             bool ok = true;
             for (int w = unit; w < p.items && ok; w += units) {
-                const int pos = item_pos(w), coff = item_coff(w);
+                const int slot = item_slot(w), coff = item_coff(w);
                 const bool half = item_half(w);
+                const int grp = slot / p.positions, pos = slot - grp * p.positions;
                 const int tm = pos / tiles_n, tn = pos % tiles_n;
                 const int row_blk = tm * NCTA + cta_rank;                 // 128-row block of S_r this CTA owns
-                for (int t = 0; t < p.terms && ok; ++t) {
+                for (int t = grp * p.terms_per_group; t < (grp + 1) * p.terms_per_group && ok; ++t) {
                     for (int ks = 0; ks < kstages; ++ks) {
                         const long long tw = TCLK();
                         if (!mbar_wait(bar_empty(stage), phase ^ 1u, ctl, 101)) { ok = false; break; }
@@ -281,7 +285,7 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                 const bool half = item_half(w);
                 // a half-width item is the same instruction with N = BN/2
                 const uint32_t idesc = half ? (idesc_full & ~(0x3Fu << 17)) | ((uint32_t)(BN >> 4) << 17) : idesc_full;
-                for (int t = 0; t < p.terms && ok; ++t) {
+                for (int t = 0; t < p.terms_per_group && ok; ++t) {
                     if (C::MX) {
                         const long long tw = TCLK();
                         if (!mbar_wait(bar_tempty(0), bphase ^ 1u, ctl, 201)) { ok = false; break; }
@@ -359,14 +363,15 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         uint32_t accu[C::MX ? C::CW : 1];               // UE8M0: raw fp32 bits drained from TMEM
         unsigned long long acc2[C::MX ? 1 : C::CW / 2]; // FP32: promoted accumulators, two columns per register pair
         for (int w = unit; w < p.items && ok; w += units) {
-            const int pos = item_pos(w), coff = item_coff(w);
+            const int slot = item_slot(w), coff = item_coff(w);
+            const int grp = slot / p.positions, pos = slot - grp * p.positions;
             const int tm = pos / tiles_n, tn = pos % tiles_n;
             const int row_in_leaf = (tm * NCTA + cta_rank) * BM + q * 32;
             // columns this warp owns: half of the item's width, in 32-column chunks
             const int cw = item_half(w) ? C::CW / 2 : C::CW;
             const int nch = cw / 32;
             const uint32_t lane_taddr = tmem_base + ((uint32_t)(q * 32) << 16) + h * cw;
-            for (int t = 0; t < p.terms && ok; ++t) {
+            for (int t = grp * p.terms_per_group; t < (grp + 1) * p.terms_per_group && ok; ++t) {
                 if (C::MX) {
                     const long long tw = TCLK();
                     if (!mbar_wait_warp(bar_tfull(0), bphase, ctl, 301)) { ok = false; break; }
@@ -607,15 +612,25 @@ fmm_status_t launch(const GemmParams& g, cudaStream_t st)
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     const int positions = (g.m / (BM * NCTA)) * (g.n / BN);
     const int max_units = sms / NCTA;
-    const int units = positions < max_units ? positions : max_units;
-    const int tail = positions % units;
+    // Term groups as separate work items only where that shortens the longest CTA's list of terms (many terms on
+    // few tile positions); otherwise one CTA (pair) walks all terms of its position.
+    int tpg = (g.terms_per_group > 0 && g.terms % g.terms_per_group == 0) ? g.terms_per_group : g.terms;
+    {
+        const long long one = (long long)((positions + max_units - 1) / max_units) * g.terms;
+        const long long many = (long long)((positions * (g.terms / tpg) + max_units - 1) / max_units) * tpg;
+        if (many >= one) tpg = g.terms;
+    }
+    const int slots = positions * (g.terms / tpg);
+    const int units = slots < max_units ? slots : max_units;
+    const int tail = slots % units;
     const bool split = C::SPLIT && tail > 0 && 2 * tail <= units;
     KParams kp;
     kp.sa = static_cast<const uint8_t*>(g.sa); kp.sb = static_cast<const uint8_t*>(g.sb);
     kp.sa_term = g.sa_term; kp.sb_term = g.sb_term;
     kp.m = g.m; kp.n = g.n; kp.k = g.k; kp.terms = g.terms;
-    kp.split_from = split ? positions - tail : positions;
-    kp.items = positions + (split ? tail : 0);
+    kp.positions = positions; kp.terms_per_group = tpg;
+    kp.split_from = split ? slots - tail : slots;
+    kp.items = slots + (split ? tail : 0);
     kp.out_start = g.out_start; kp.out = g.out; kp.status = g.status;
 
     cudaLaunchConfig_t cfg;

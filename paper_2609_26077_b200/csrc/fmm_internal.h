@@ -97,6 +97,7 @@ struct GemmParams {
     int m, n, k, terms;
     const int* out_start; const FmmOutEntry* out;
     int* status;
+    int terms_per_group;                    // consecutive terms that feed the same output blocks (R at levels >= 2, else all)
     int sb_tile;                            // fp32 scales, blk 128: the B-side scale is constant over each 128-column tile
 };
 fmm_status_t fmm_launch_bounded_wait_selftest(int* status, unsigned long long limit_ns, cudaStream_t st);
