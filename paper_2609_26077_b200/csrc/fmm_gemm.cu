@@ -37,7 +37,7 @@ constexpr int MODE_FP32_SB_TILE = 2;
 constexpr int BM = 128;                 // rows per CTA
 constexpr int BK = 128;                 // K elements (= bytes) per pipeline stage: one swizzle row
 constexpr int EPI_WARPS = 8;               // two per TMEM lane quadrant, each half of the tile's columns
-constexpr int EPI_WARP0 = 4;               // warps 0..3: producer, MMA issuer, two idle (one warpgroup)
+constexpr int EPI_WARP0 = 4;               // warps 0..3: operand producer, MMA issuer, scale producer (FP32 modes), idle
 constexpr int NUM_THREADS = (EPI_WARP0 + EPI_WARPS) * 32;
 // setmaxnreg budget: the CTA's register pool is NUM_THREADS x (registers at launch); an increase
 // beyond what the decrease freed would block forever, so the split is checked here.
@@ -224,7 +224,6 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
             int stage = 0; uint32_t phase = 0;
-            int ss = 0; uint32_t sphase = 0;
             bool ok = true;
             for (int w = unit; w < p.items && ok; w += units) {
                 const int slot = item_slot(w), coff = item_coff(w);
@@ -232,7 +231,8 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                 const int grp = slot / p.positions, pos = slot - grp * p.positions;
                 const int tm = pos / tiles_n, tn = pos % tiles_n;
                 const int row_blk = tm * NCTA + cta_rank;                 // 128-row block of S_r this CTA owns
-                for (int t = grp * p.terms_per_group; t < (grp + 1) * p.terms_per_group && ok; ++t) {
+                const int t_end = (grp + 1) * p.terms_per_group;
+                for (int t = t_end - p.terms_per_group; t < t_end && ok; ++t) {
                     for (int ks = 0; ks < kstages; ++ks) {
                         const long long tw = TCLK();
                         if (!mbar_wait(bar_empty(stage), phase ^ 1u, ctl, 101)) { ok = false; break; }
@@ -255,18 +255,34 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                                 tma_load_2d<NCTA>(sf + 512, &tmSFB, 0, (t * (nkb >> 2) + ks) * row_blocks_b + tn * C::SFB_ATOMS, fb);
                             else
                                 tma_load_2d<NCTA>(sf + 512, &tmSFBh, 0, (t * (nkb >> 2) + ks) * row_blocks_b + tn * C::SFB_ATOMS + coff / 128, fb);
-                        } else {
-                            if (!mbar_wait(bar_sempty(ss), sphase ^ 1u, ctl, 102)) { ok = false; break; }
-                            mbar_expect_tx(bar_sfull(ss), C::SB_STAGE_BYTES);
-#pragma unroll
-                            for (int g = 0; g < C::KB_PER_STAGE; ++g) {
-                                const uint8_t* gb = p.sb + (long long)t * p.sb_term +
-                                                    ((long long)(ks * C::KB_PER_STAGE + g) * p.n + tn * BN) * 4;
-                                bulk_load(base + C::OFF_SB + ss * C::SB_STAGE_BYTES + g * BN * 4, gb, BN * 4, bar_sfull(ss));
-                            }
-                            if (++ss == C::SB_STAGES) { ss = 0; sphase ^= 1u; }
                         }
                         if (++stage == C::STAGES) { stage = 0; phase ^= 1u; }
+                    }
+                }
+            }
+        }
+    } else if (warp == 2) {
+        // ------------------------------------------------------------------ FP32 modes: producer of the B-side scales
+        // (its own thread and ring: the operand producer above has no registers to spare, and the scale ring is
+        // released by the promoting warps, not by the tensor pipe)
+        if (!C::MX && lane == 0) {
+            int ss = 0; uint32_t sphase = 0;
+            bool ok = true;
+            for (int w = unit; w < p.items && ok; w += units) {
+                const int slot = item_slot(w);
+                const int grp = slot / p.positions, pos = slot - grp * p.positions;
+                const int tn = pos % tiles_n;
+                const int t_end = (grp + 1) * p.terms_per_group;
+                for (int t = t_end - p.terms_per_group; t < t_end && ok; ++t) {
+                    const uint8_t* sb_t = p.sb + (long long)t * p.sb_term + (long long)tn * BN * 4;
+                    for (int ks = 0; ks < kstages; ++ks) {
+                        if (!mbar_wait(bar_sempty(ss), sphase ^ 1u, ctl, 102)) { ok = false; break; }
+                        mbar_expect_tx(bar_sfull(ss), C::SB_STAGE_BYTES);
+#pragma unroll
+                        for (int g = 0; g < C::KB_PER_STAGE; ++g)
+                            bulk_load(base + C::OFF_SB + ss * C::SB_STAGE_BYTES + g * BN * 4,
+                                      sb_t + (long long)(ks * C::KB_PER_STAGE + g) * p.n * 4, BN * 4, bar_sfull(ss));
+                        if (++ss == C::SB_STAGES) { ss = 0; sphase ^= 1u; }
                     }
                 }
             }
@@ -356,10 +372,6 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         int ss = 0; uint32_t sphase = 0;
         uint32_t store_cnt = 0;
         bool ok = true;
-        // Each C tile is updated once per term that feeds it, and between two updates a whole term's operands
-        // stream through L2: the tiles are marked evict-last (at n = 8192: fewer write-backs of half-accumulated
-        // tiles, product kernel 3 % faster; an evict-first policy on the operand loads was slower).
-        const uint64_t pol_c = policy_evict_last();
         uint32_t accu[C::MX ? C::CW : 1];               // UE8M0: raw fp32 bits drained from TMEM
         unsigned long long acc2[C::MX ? 1 : C::CW / 2]; // FP32: promoted accumulators, two columns per register pair
         for (int w = unit; w < p.items && ok; w += units) {
@@ -371,7 +383,7 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             const int cw = item_half(w) ? C::CW / 2 : C::CW;
             const int nch = cw / 32;
             const uint32_t lane_taddr = tmem_base + ((uint32_t)(q * 32) << 16) + h * cw;
-            for (int t = grp * p.terms_per_group; t < (grp + 1) * p.terms_per_group && ok; ++t) {
+            for (int t = grp * p.terms_per_group, left = p.terms_per_group; left > 0 && ok; ++t, --left) {
                 if (C::MX) {
                     const long long tw = TCLK();
                     if (!mbar_wait_warp(bar_tfull(0), bphase, ctl, 301)) { ok = false; break; }
@@ -474,6 +486,11 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                 }
                 // ---- post-addition: W-weighted scatter of this product into its C blocks
                 const long long t_out = TCLK();
+                // Each C tile is updated once per term that feeds it, and between two updates a whole term's operands
+                // stream through L2: the tiles are marked evict-last (at n = 8192: fewer write-backs of
+                // half-accumulated tiles, product kernel 3 % faster; evict-first on the operand loads was slower).
+                // The policy word is rebuilt here so that it is not live across the promotion loop.
+                const uint64_t pol_c = policy_evict_last();
                 const int o0 = p.out_start[t], o1 = p.out_start[t + 1];
                 if (lane == 0) bulk_wait<0>();     // the previous term's writes to these tiles have landed
                 __syncwarp();
