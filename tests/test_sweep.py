@@ -33,7 +33,7 @@ def test_summarise_pairs_ratios_and_pools(tmp_path):
 def test_config_c1_on_gpu(tmp_path):
     import argparse
     out = tmp_path / "c1.jsonl"
-    args = argparse.Namespace(config="c1", scale_mode="fp32", block_k=32, out=str(out), trials=6)
+    args = argparse.Namespace(config="c1", scale_mode="fp32", block_k=32, out=str(out), trials=6, b_tile=0, b_bf16=False)
     sweep.run(args)
     n_lines = len(out.read_text().splitlines())
     assert n_lines == 12
