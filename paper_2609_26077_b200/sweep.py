@@ -188,6 +188,52 @@ def orbit_stability(path, file=sys.stdout):
     return out
 
 
+def covariance_diagnostic(names=("strassen", "winograd", "phi_optimal", "strassen_rb", "winograd_rb", "phi_optimal_rb"),
+                          n=512, seeds=4, block_k=128, scale_mode="fp32", family="gaussian", file=sys.stdout):
+    """Cross-term covariance diagnostic (App. D.1): the part of the error that is linear in the rounding
+    residuals is L_q = sum_r W[r][q] t_r with t_r = dx_r y_r + x_r dy_r (x_r, y_r the encoded combinations,
+    dx_r, dy_r their quantization residuals).  The model keeps only the diagonal sum_{r,q} W[r][q]^2 |t_r|_F^2
+    (that is what defines Phi); the fraction (|L|_F^2 - diag) / |L|_F^2 measures what the dropped cross terms
+    contribute.  The quantized operands come from the CUDA encoder; the algebra around them is fp64 numpy.
+    The paper reports armwise means between -0.085 % and 0.201 % (n = 512, Gaussian, four seeds, 1 x 128 groups)."""
+    import torch
+    rows = []
+    for name in names:
+        U, V, W = (np.asarray(x, dtype=np.float64) for x in P.get(name))
+        plan = fmm.Plan(*P.get(name), levels=1, block_k=block_k, scale_mode=scale_mode)
+        fr = []
+        for seed in range(seeds):
+            A, B = Wl.FAMILIES[family](n, n, n, seed)
+            ws = plan.workspace(n, n, n)
+            plan.encode_only(torch.from_numpy(A).cuda(), torch.from_numpy(B).cuda(), workspace=ws)
+            torch.cuda.synchronize()
+            h = n // 2
+            Aq = [A[:h, :h], A[:h, h:], A[h:, :h], A[h:, h:]]
+            Bq = [B[:h, :h], B[:h, h:], B[h:, :h], B[h:, h:]]
+            t = []
+            for r in range(U.shape[0]):
+                x = sum(U[r, j] * Aq[j].astype(np.float64) for j in range(4))
+                y = sum(V[r, j] * Bq[j].astype(np.float64) for j in range(4))
+                ca, sa = plan.quantized_operand(ws, n, n, n, r, "A")
+                cb, sb = plan.quantized_operand(ws, n, n, n, r, "B")
+                if scale_mode != "fp32":
+                    sa, sb = np.ldexp(1.0, sa.astype(np.int32) - 127), np.ldexp(1.0, sb.astype(np.int32) - 127)
+                dec = torch.arange(256, dtype=torch.uint8).view(torch.float8_e4m3fn).to(torch.float64).numpy()
+                xh = dec[ca] * np.repeat(sa.astype(np.float64), block_k, axis=1)
+                yh = dec[cb] * np.repeat(sb.astype(np.float64), block_k, axis=0)
+                t.append((xh - x) @ y + x @ (yh - y))
+            Lsq = sum(np.linalg.norm(sum(W[r, q] * t[r] for r in range(len(t)))) ** 2 for q in range(4))
+            diag = sum(W[r, q] ** 2 * np.linalg.norm(t[r]) ** 2 for r in range(len(t)) for q in range(4))
+            fr.append((Lsq - diag) / Lsq)
+        plan.close()
+        rows.append((name, float(np.mean(fr)), float(np.min(fr)), float(np.max(fr))))
+    print(f"| realization | mean residual fraction | min | max |  (n = {n}, {family}, {seeds} seeds, {scale_mode} blk {block_k})", file=file)
+    print("|---|---|---|---|", file=file)
+    for name, m, lo, hi in rows:
+        print(f"| {name} | {100 * m:+.3f} % | {100 * lo:+.3f} % | {100 * hi:+.3f} % |", file=file)
+    return rows
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--config", choices=sorted(CONFIGS))
@@ -200,6 +246,7 @@ def main():
     ap.add_argument("--summarise")
     ap.add_argument("--ladder", help="panel statistics of a c7 output file")
     ap.add_argument("--orbit", help="orbit-ratio stability of a c8 output file")
+    ap.add_argument("--covariance", action="store_true", help="cross-term covariance diagnostic (n = 512, four seeds)")
     a = ap.parse_args()
     if a.summarise:
         summarise(a.summarise)
@@ -207,6 +254,8 @@ def main():
         ladder_summary(a.ladder)
     elif a.orbit:
         orbit_stability(a.orbit)
+    elif a.covariance:
+        covariance_diagnostic(block_k=a.block_k, scale_mode=a.scale_mode)
     else:
         if not a.config:
             ap.error("--config or --summarise is required")

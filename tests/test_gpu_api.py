@@ -92,3 +92,29 @@ def test_bounded_wait_runs_out_and_leaves_the_context_usable():
     want = O.fused_fmm(A, B, *P.get("strassen"), levels=1, blk=32, mode=O.SCALE_UE8M0)
     assert np.linalg.norm(got - want) / np.linalg.norm(want) < 1e-5
     assert plan.device_status() == (0, 0)
+
+
+def test_matmul_can_be_captured_in_a_cuda_graph():
+    # fmm_matmul allocates nothing and never synchronises with the host, so the whole path (encode, products,
+    # decode; here two recursion levels = 5 launches) can be captured once and replayed
+    M, K, N = 512, 512, 512
+    A, B = Wl.gaussian(M, K, N, 21)
+    a, b = dev(A), dev(B)
+    for mode in ("fp32", "ue8m0"):
+        plan = make_plan("phi_optimal", 2, 32, mode)
+        ws = plan.workspace(M, N, K)
+        eager = plan.matmul(a, b, workspace=ws).clone()          # also warms up (function attributes are set once)
+        out = torch.zeros((M, N), device="cuda")
+        stream = torch.cuda.Stream()
+        stream.wait_stream(torch.cuda.current_stream())
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(stream):
+            with torch.cuda.graph(graph, stream=stream):
+                plan.matmul(a, b, out=out, workspace=ws, stream=stream)
+        torch.cuda.current_stream().wait_stream(stream)
+        for _ in range(3):
+            out.fill_(float("nan"))
+            graph.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(out, eager)
+        assert plan.device_status() == (0, 0)

@@ -43,3 +43,11 @@ def test_config_c1_on_gpu(tmp_path):
     by = {(r[1], r[2]): r for r in rows}
     assert by[("cubic", 0)][4] == pytest.approx(0.0339, rel=0.03)
     assert by[("strassen", 1)][7] == pytest.approx(2.0, rel=0.03)
+
+
+@pytest.mark.gpu
+def test_covariance_diagnostic_is_small_on_gaussian_operands():
+    # App. D.1: the cross-r part of the linear error term is a fraction of a percent of the whole
+    rows = sweep.covariance_diagnostic(names=("strassen", "phi_optimal"), n=256, seeds=2, block_k=128, file=io.StringIO())
+    for name, mean, lo, hi in rows:
+        assert abs(mean) < 0.03 and lo > -0.06 and hi < 0.06, (name, mean, lo, hi)
