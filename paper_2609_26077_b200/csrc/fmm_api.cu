@@ -65,8 +65,12 @@ void make_layout(const fmm_plan* plan, int64_t M, int64_t N, int64_t K, FmmLayou
     for (int lv = 1; lv < plan->levels; ++lv) {
         const int64_t cnt = fmm_ipow(plan->rank, lv);
         const int64_t dd = (int64_t)1 << lv;
-        L->inter_a[lv] = off; off = align_up(off + (size_t)(cnt * (M / dd) * (K / dd)) * 4, 1024);
-        L->inter_b[lv] = off; off = align_up(off + (size_t)(cnt * (K / dd) * (N / dd)) * 4, 1024);
+        // the innermost of these levels is formed in registers by the two-level encoder where that exists
+        const bool last = (lv == plan->levels - 1);
+        const bool need_a = !(last && fmm_encode2_supported(false, plan->qp.block_k, 0, 0));
+        const bool need_b = !(last && fmm_encode2_supported(true, plan->qp.block_k, plan->qp.b_tile_n, plan->qp.b_preround_bf16));
+        if (need_a) { L->inter_a[lv] = off; off = align_up(off + (size_t)(cnt * (M / dd) * (K / dd)) * 4, 1024); }
+        if (need_b) { L->inter_b[lv] = off; off = align_up(off + (size_t)(cnt * (K / dd) * (N / dd)) * 4, 1024); }
         L->dec[lv] = off; off = align_up(off + (size_t)(cnt * (M / dd) * (N / dd)) * 4, 1024);
     }
     L->total = off;
