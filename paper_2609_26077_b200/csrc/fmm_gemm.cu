@@ -54,7 +54,12 @@ struct Cfg {
     // The UE8M0 pair kernel is bound by operand-load latency under L2 contention: it trades epilogue
     // staging space for more pipeline stages.
     static constexpr int STAGING_BUFS = (MX && NCTA == 2) ? 1 : 2;
-    static constexpr int STAGES = (MX && NCTA == 2) ? 6 : ((A_BYTES + B_BYTES) > 40000 ? 3 : 4);
+    static constexpr bool DUMP = !MX && BN == 128 && BK / BLK == 4;
+    static constexpr int STAGES = (MX && NCTA == 2) ? 6 : ((A_BYTES + B_BYTES) > 40000 || DUMP ? 3 : 4);
+    // FP32 scales, block 32 (DUMP, above): the promoting warps hand a finished product to a dedicated output warp
+    // through a shared-memory copy of the (unweighted) accumulators and go straight on with the next term; the
+    // W-weighted stores / add-reductions then overlap the next term's promotion instead of stalling it.
+    static constexpr int DUMP_BYTES = DUMP ? BM * BN * 4 : 0;
     // output chunk of one epilogue warp: 32 rows x CH fp32, staged in shared memory for one TMA store
     // (the UE8M0 pair kernel halves it: with one narrow buffer per warp a sixth operand stage fits)
     static constexpr int CH = (MX && NCTA == 2) ? 16 : 32;
@@ -69,10 +74,12 @@ struct Cfg {
     static constexpr int OFF_A = 0;
     static constexpr int OFF_B = OFF_A + STAGES * A_BYTES;
     static constexpr int OFF_STG = OFF_B + STAGES * B_BYTES;
-    static constexpr int OFF_SF = OFF_STG + EPI_WARPS * STAGING_BUFS * STAGING_BYTES;
+    static constexpr int OUT_BUFS = 8;          // DUMP: staging chunks of the output warp (TMA stores in flight)
+    static constexpr int OFF_DUMP = OFF_STG + (DUMP ? OUT_BUFS * 4096 : EPI_WARPS * STAGING_BUFS * STAGING_BYTES);
+    static constexpr int OFF_SF = OFF_DUMP + DUMP_BYTES;
     static constexpr int OFF_SB = OFF_SF + STAGES * SF_STAGE_BYTES;
     static constexpr int OFF_BAR = OFF_SB + SB_STAGES * SB_STAGE_BYTES;
-    static constexpr int NUM_BARS = 2 * STAGES + 2 * SB_STAGES + 8;
+    static constexpr int NUM_BARS = 2 * STAGES + 2 * SB_STAGES + 8 + 2;
     static constexpr int SMEM_BYTES = OFF_BAR + NUM_BARS * 8 + 16 + 1024;   // + alignment slack
     // TMEM: MX: one BN-column accumulator, then per stage 4 SFA + 4*(BN/128) SFB columns.
     //       FP32: ring of 512/BN accumulators, one per K block in flight.
@@ -178,6 +185,8 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     auto bar_sempty = [&](int s) { return bar0 + 8u * (2 * C::STAGES + C::SB_STAGES + s); };
     auto bar_tfull = [&](int b) { return bar0 + 8u * (2 * C::STAGES + 2 * C::SB_STAGES + b); };
     auto bar_tempty = [&](int b) { return bar0 + 8u * (2 * C::STAGES + 2 * C::SB_STAGES + 4 + b); };
+    const uint32_t bar_dfull = bar0 + 8u * (2 * C::STAGES + 2 * C::SB_STAGES + 8);      // accumulator copy written
+    const uint32_t bar_dempty = bar_dfull + 8u;                                           // ... and consumed
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base_ptr + C::OFF_BAR + C::NUM_BARS * 8);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
     const Ctl ctl{abort_flag, p.status};
@@ -196,6 +205,7 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         for (int s = 0; s < C::STAGES; ++s) { mbar_init(bar_full(s), 1); mbar_init(bar_empty(s), 1); }
         for (int s = 0; s < C::SB_STAGES; ++s) { mbar_init(bar_sfull(s), 1); mbar_init(bar_sempty(s), EPI_WARPS); }
         for (int b = 0; b < 4; ++b) { mbar_init(bar_tfull(b), 1); mbar_init(bar_tempty(b), NCTA * EPI_WARPS); }
+        mbar_init(bar_dfull, EPI_WARPS); mbar_init(bar_dempty, 1);
         *abort_flag = 0;
         fence_barrier_init();
     }
@@ -287,6 +297,76 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                 }
             }
         }
+    } else if (warp == 3) {
+        // ------------------------------------------------------------------ FP32 modes, 128-column tiles: output warp
+        if (C::DUMP) {
+            const uint32_t stg = base + C::OFF_STG + lane * 128;          // this lane's row of a staging chunk
+            const uint32_t dump = base + C::OFF_DUMP + lane * 128;        // ... and of a chunk of the accumulator copy
+            uint32_t dphase = 0, store_cnt = 0;
+            bool ok = true;
+            for (int w = unit; w < p.items && ok; w += units) {
+                const int slot = item_slot(w);
+                const int grp = slot / p.positions, pos = slot - grp * p.positions;
+                const int tm = pos / tiles_n, tn = pos % tiles_n;
+                const int t_end = (grp + 1) * p.terms_per_group;
+                for (int t = t_end - p.terms_per_group; t < t_end && ok; ++t) {
+                    if (!mbar_wait_warp(bar_dfull, dphase, ctl, 401)) { ok = false; break; }
+                    dphase ^= 1u;
+                    const int o0 = p.out_start[t], o1 = p.out_start[t + 1];
+                    if (lane == 0) bulk_wait<0>();     // the previous term's writes to these tiles have landed
+                    __syncwarp();
+                    for (int o = o0; o < o1; ++o) {
+                        const FmmOutEntry ent = p.out[o];
+                        const int row0 = ent.row_off * p.m + (tm * NCTA + cta_rank) * BM;
+                        const int col0 = ent.col_off * p.n + tn * BN;
+#pragma unroll 1
+                        for (int ch0 = 0; ch0 < (BM / 32) * (BN / 32); ch0 += C::OUT_BUFS / 2) {
+                            // OUT_BUFS/2 chunks of 32 rows x 32 columns per round (one proxy fence and one bulk group per
+                            // round, two rounds in flight).  The promoting warps stored the chunks in the swizzled layout
+                            // the tensor map expects; they are copied through registers to apply the weight.
+                            const uint32_t b0 = (store_cnt & 1u) * (C::OUT_BUFS / 2);
+                            if (lane == 0) bulk_wait_read<1>();
+                            __syncwarp();
+#pragma unroll 1
+                            for (int k = 0; k < C::OUT_BUFS / 2; ++k) {
+                                const uint32_t src = dump + (ch0 + k) * 4096;
+                                const uint32_t dst = stg + (b0 + k) * 4096;
+#pragma unroll 1
+                                for (int i0 = 0; i0 < 8; i0 += 4) {      // four 16-byte pieces at a time: this warp has 56 registers
+#pragma unroll
+                                    for (int i4 = i0; i4 < i0 + 4; ++i4) {
+                                        // same physical piece on both sides (the swizzle is kept); the lane-dependent
+                                        // order only spreads the 32 rows over the shared-memory banks
+                                        const int pc = (i4 ^ (lane & 7)) << 4;
+                                        float4 v = lds128(src + pc);
+                                        v.x *= ent.w; v.y *= ent.w; v.z *= ent.w; v.w *= ent.w;
+                                        sts128(dst + pc, v);
+                                    }
+                                }
+                            }
+                            fence_proxy_async();
+                            __syncwarp();
+                            if (lane == 0) {
+                                const uint64_t pol_c = policy_evict_last();     // see the note on the C tiles' L2 policy below
+#pragma unroll 1
+                                for (int k = 0; k < C::OUT_BUFS / 2; ++k) {
+                                    const int ch = ch0 + k;
+                                    const int r = row0 + (ch / (BN / 32)) * 32, c = col0 + (ch % (BN / 32)) * 32;
+                                    if (ent.first) tma_store_2d_hint(&tmC, c, r, stg + (b0 + k) * 4096, pol_c);      // lane 0: stg = chunk base
+                                    else tma_reduce_add_2d_hint(&tmC, c, r, stg + (b0 + k) * 4096, pol_c);
+                                }
+                                bulk_commit();
+                            }
+                            ++store_cnt;
+                        }
+                    }
+                    // every lane has read the copy for the last time
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar_dempty);
+                }
+            }
+            if (lane == 0) bulk_wait<0>();
+        }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer (even CTA only in a pair)
         if (lane == 0 && leader) {
@@ -371,6 +451,7 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         int buf = 0; uint32_t bphase = 0;
         int ss = 0; uint32_t sphase = 0;
         uint32_t store_cnt = 0;
+        uint32_t dphase = 0;
         bool ok = true;
         uint32_t accu[C::MX ? C::CW : 1];               // UE8M0: raw fp32 bits drained from TMEM
         unsigned long long acc2[C::MX ? 1 : C::CW / 2]; // FP32: promoted accumulators, two columns per register pair
@@ -483,6 +564,27 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                         if (++ss == C::SB_STAGES) { ss = 0; sphase ^= 1u; }
                     }
                     if (!ok) break;
+                }
+                if (C::DUMP) {
+                    // ---- hand the finished product to the output warp: rows q*32 + lane, columns h*CW .. of the tile,
+                    // as 32 x 32 chunks in the 128-byte-swizzled layout of the output tensor map
+                    const long long t_dump = TCLK();
+                    if (!mbar_wait_warp(bar_dempty, dphase ^ 1u, ctl, 304)) { ok = false; break; }
+                    dphase ^= 1u;
+                    uint8_t* dptr = base_ptr + C::OFF_DUMP + (q * (BN / 32) + h * (C::CW / 32)) * 4096 + lane * 128;
+#pragma unroll
+                    for (int c = 0; c < C::CW / 32; ++c)
+#pragma unroll
+                        for (int i4 = 0; i4 < 8; ++i4) {
+                            float4 v;
+                            unpack2(acc2[c * 16 + i4 * 2], v.x, v.y);
+                            unpack2(acc2[c * 16 + i4 * 2 + 1], v.z, v.w);
+                            *reinterpret_cast<float4*>(dptr + c * 4096 + ((i4 ^ (lane & 7)) << 4)) = v;
+                        }
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar_dfull);
+                    TADD(4, t_dump);
+                    continue;
                 }
                 // ---- post-addition: W-weighted scatter of this product into its C blocks
                 const long long t_out = TCLK();
