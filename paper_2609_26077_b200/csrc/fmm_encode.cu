@@ -567,14 +567,10 @@ __global__ void __launch_bounds__(256) decode_kernel(const DecodeParams p)
 
 int sm_count()
 {
-    static int n = 0;
-    if (!n) {
-        int dev = 0;
-        cudaGetDevice(&dev);
-        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
-        if (n <= 0) n = 148;
-    }
-    return n;
+    int dev = 0, n = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);      // a cached host-side attribute: cheap
+    return n > 0 ? n : 148;
 }
 
 }  // namespace

@@ -23,6 +23,7 @@
 //
 // Every wait is bounded: on time-out a status word is set and all roles leave the kernel.
 #include <string.h>
+#include <atomic>
 #include "fmm_internal.h"
 #include "fmm_ptx.cuh"
 
@@ -718,17 +719,18 @@ fmm_status_t launch(const GemmParams& g, cudaStream_t st)
         if (!make_map_2d(&tmBh, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, g.qb, (uint64_t)g.k, (uint64_t)g.terms * g.n, BK, C::BROWS / 2, SW)) return FMM_ERR_CUDA;
         if (!make_map_2d(&tmSFBh, CU_TENSOR_MAP_DATA_TYPE_UINT32, 4, g.sb, 128, atoms_b, 128, 1, CU_TENSOR_MAP_SWIZZLE_NONE)) return FMM_ERR_CUDA;
     }
-    static bool attr_set = false;
-    if (!attr_set) {
+    int dev = 0, sms = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    // the dynamic shared memory limit is a per-device attribute of the function: set once per device
+    static std::atomic<bool> attr_set[64];
+    if (dev < 0 || dev >= 64 || !attr_set[dev].load(std::memory_order_acquire)) {
         if (cudaFuncSetAttribute(fmm_gemm_kernel<BN, MODE, BLK, NCTA>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES) != cudaSuccess) {
             cudaGetLastError();
             return FMM_ERR_CUDA;
         }
-        attr_set = true;
+        if (dev >= 0 && dev < 64) attr_set[dev].store(true, std::memory_order_release);
     }
-    int dev = 0, sms = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     const int positions = (g.m / (BM * NCTA)) * (g.n / BN);
     const int max_units = sms / NCTA;
     // Term groups as separate work items only where that shortens the longest CTA's list of terms (many terms on
