@@ -34,6 +34,12 @@ using namespace fmmptx;
 // 128-column tile (the 128 x 128 weight tiles of App. E.5).  The promotion then needs one multiply per row
 // and K block (s = sA * sB_tile) and one FMA per element, instead of a multiply and an FMA per element.
 constexpr int MODE_FP32_SB_TILE = 2;
+// Internal fourth mode: FP32 scales (per column, as mode 0) with a dedicated output warp.  The promoting warps hand
+// a finished product to it through a shared-memory copy of the (unweighted) accumulators and go straight on with
+// the next term; the W-weighted stores / add-reductions then overlap the next term's promotion instead of stalling
+// it.  The output warp needs a fixed time per term, so this pays only when a term has many K stages (measured
+// cross-over between 16 and 32 stages of 128 k); the dispatcher picks the mode per launch.
+constexpr int MODE_FP32_OUT_WARP = 3;
 
 constexpr int BM = 128;                 // rows per CTA
 constexpr int BK = 128;                 // K elements (= bytes) per pipeline stage: one swizzle row
@@ -55,11 +61,10 @@ struct Cfg {
     // The UE8M0 pair kernel is bound by operand-load latency under L2 contention: it trades epilogue
     // staging space for more pipeline stages.
     static constexpr int STAGING_BUFS = (MX && NCTA == 2) ? 1 : 2;
-    static constexpr bool DUMP = !MX && BN == 128 && BK / BLK == 4;
+    static constexpr bool DUMP = (MODE == MODE_FP32_OUT_WARP);
+    static_assert(!DUMP || (BN == 128 && BK / BLK == 4), "output-warp mode: 128-column tiles, block 32");
     static constexpr int STAGES = (MX && NCTA == 2) ? 6 : ((A_BYTES + B_BYTES) > 40000 || DUMP ? 3 : 4);
-    // FP32 scales, block 32 (DUMP, above): the promoting warps hand a finished product to a dedicated output warp
-    // through a shared-memory copy of the (unweighted) accumulators and go straight on with the next term; the
-    // W-weighted stores / add-reductions then overlap the next term's promotion instead of stalling it.
+    // DUMP (output-warp mode): shared-memory copy of a finished product, BM x BN fp32
     static constexpr int DUMP_BYTES = DUMP ? BM * BN * 4 : 0;
     // output chunk of one epilogue warp: 32 rows x CH fp32, staged in shared memory for one TMA store
     // (the UE8M0 pair kernel halves it: with one narrow buffer per warp a sixth operand stage fits)
@@ -334,14 +339,16 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                                 const uint32_t dst = stg + (b0 + k) * 4096;
 #pragma unroll 1
                                 for (int i0 = 0; i0 < 8; i0 += 4) {      // four 16-byte pieces at a time: this warp has 56 registers
+                                    // same physical piece on both sides (the swizzle is kept); the lane-dependent order
+                                    // only spreads the 32 rows over the shared-memory banks.  All four loads are issued
+                                    // before the first store.
+                                    float4 v[4];
 #pragma unroll
-                                    for (int i4 = i0; i4 < i0 + 4; ++i4) {
-                                        // same physical piece on both sides (the swizzle is kept); the lane-dependent
-                                        // order only spreads the 32 rows over the shared-memory banks
-                                        const int pc = (i4 ^ (lane & 7)) << 4;
-                                        float4 v = lds128(src + pc);
-                                        v.x *= ent.w; v.y *= ent.w; v.z *= ent.w; v.w *= ent.w;
-                                        sts128(dst + pc, v);
+                                    for (int i4 = 0; i4 < 4; ++i4) v[i4] = lds128(src + (((i0 + i4) ^ (lane & 7)) << 4));
+#pragma unroll
+                                    for (int i4 = 0; i4 < 4; ++i4) {
+                                        v[i4].x *= ent.w; v[i4].y *= ent.w; v[i4].z *= ent.w; v[i4].w *= ent.w;
+                                        sts128(dst + (((i0 + i4) ^ (lane & 7)) << 4), v[i4]);
                                     }
                                 }
                             }
@@ -781,6 +788,12 @@ fmm_status_t launch_shape(const GemmParams& g, cudaStream_t st)
             // one promotion per 128 k: the tensor pipe matters again, and 256-column instructions read half as
             // much shared memory per flop as 128-column ones
             if ((g.m % 256) == 0 && (g.n % 256) == 0) return launch<256, MODE, BLK, 2>(g, st);
+        }
+        if constexpr (BLK == 32 && MODE == FMM_SCALE_FP32_AMAX_DIV_448) {
+            if (g.k / BK >= 24) {           // long terms: post-addition by the output warp
+                if ((g.m % 256) == 0) return launch<128, MODE_FP32_OUT_WARP, BLK, 2>(g, st);
+                return launch<128, MODE_FP32_OUT_WARP, BLK, 1>(g, st);
+            }
         }
         if ((g.m % 256) == 0) return launch<128, MODE, BLK, 2>(g, st);
         return launch<128, MODE, BLK, 1>(g, st);
