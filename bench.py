@@ -39,6 +39,7 @@ def parse():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--n", type=int, default=8192)
+    ap.add_argument("--shape", default="", help="M,K,N of a rectangular problem (profiling captures); overrides --n")
     ap.add_argument("--levels", type=int, default=1)
     ap.add_argument("--realization", default="phi_optimal")
     ap.add_argument("--scale-mode", default="fp32", choices=["fp32", "ue8m0"])
@@ -156,6 +157,8 @@ def run_ours(args):
 
     n, K_steps, W_steps = args.n, args.steps, max(args.warmup, 3)
     M = N = K = n
+    if args.shape:
+        M, K, N = (int(x) for x in args.shape.split(","))
     pk = peaks()
     gen = torch.Generator(device="cuda")
     gen.manual_seed(1234 + rank_id)
@@ -240,9 +243,10 @@ def run_ours(args):
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K_steps, "warmup": W_steps,
         "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "fp8_e4m3", "data": "synthetic",
-        "config": {"workload": f"n={n} square, {args.levels} level(s), {args.realization}, A,B iid N(0,1) fp32 (BASELINE configs[2])",
+        "config": {"workload": (f"n={n} square" if not args.shape else f"M,K,N={M},{K},{N}") +
+                               f", {args.levels} level(s), {args.realization}, A,B iid N(0,1) fp32 (BASELINE configs[2])",
                    "scale_mode": args.scale_mode, "block_k": args.block_k, "M": M, "N": N, "K": K,
-                   "l2": "inputs larger than L2 (2 x 268 MB fp32 operands, 268 MB output)",
+                   "l2": f"inputs larger than L2 ({4 * M * K / 1e6:.0f} + {4 * K * N / 1e6:.0f} MB fp32 operands, {4 * M * N / 1e6:.0f} MB output)",
                    "multi_gpu": "replicas only"},
         "clocks": clocks,
         "gpu_launches": launches_per_step * K_steps,
