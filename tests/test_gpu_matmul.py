@@ -82,6 +82,18 @@ def test_repeat_calls_are_bit_reproducible_and_overwrite_c():
     assert torch.equal(c1, out)
 
 
+def test_output_warp_variant_is_bit_reproducible():
+    # 48 K stages per term: the fp32 / block-32 product runs the kernel variant whose post-addition is issued by a
+    # dedicated warp while the next term is being promoted; the order of the add-reductions per tile is still fixed
+    A, B = Wl.llm_shaped(512, 12288, 512, 2)
+    plan = make_plan("phi_optimal", 1, 32, "fp32")
+    a, b = dev(A), dev(B)
+    c1 = plan.matmul(a, b).clone()
+    for _ in range(3):
+        assert torch.equal(plan.matmul(a, b), c1)
+    assert plan.device_status() == (0, 0)
+
+
 def test_errors_vs_fp64_reference_match_oracle_ratios():
     # the measured RMS error ratios between realizations must match the oracle's within 2 %
     n, seeds = 512, range(4)
