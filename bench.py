@@ -307,6 +307,35 @@ def run_ours(args):
                              "ms_per_step": ms, "value": flop_eff / (ms * 1e-3) / 1e12})
             p2.close()
         out["variants"] = variants
+        # the paper's timing protocol (App. E.7): interleaved repetitions across realizations, median and a
+        # bootstrap 95 % interval of the median, so that clock drift hits every arm alike
+        arms = [("cubic", 0), ("strassen", 1), ("phi_optimal", 1)]
+        plans = [(nm, make_plan(nm, lv, args.block_k, args.scale_mode)) for nm, lv in arms]
+        wss = [pl.workspace(M, N, K) for _, pl in plans]
+        for (_, pl), w2 in zip(plans, wss):
+            for _ in range(5):
+                pl.matmul(A, B, out=C, workspace=w2)
+        torch.cuda.synchronize()
+        samples = {nm: [] for nm, _ in arms}
+        for _ in range(25):
+            for (nm, pl), w2 in zip(plans, wss):
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                pl.matmul(A, B, out=C, workspace=w2)
+                e1.record()
+                e1.synchronize()
+                samples[nm].append(e0.elapsed_time(e1))
+        import numpy as _np
+        rng = _np.random.default_rng(0)
+        inter = {}
+        for nm, xs in samples.items():
+            xs = _np.array(xs)
+            boot = _np.median(rng.choice(xs, size=(2000, xs.size), replace=True), axis=1)
+            inter[nm] = {"median_ms": float(_np.median(xs)), "ci95_ms": [float(_np.percentile(boot, 2.5)), float(_np.percentile(boot, 97.5))],
+                         "value": flop_eff / (float(_np.median(xs)) * 1e-3) / 1e12}
+        out["interleaved"] = {"repetitions": 25, "scale_mode": args.scale_mode, "block_k": args.block_k, "arms": inter}
+        for _, pl in plans:
+            pl.close()
         # RMS relative error vs the fp64 product, and ratios vs cubic fp8 in the same quantizer
         ref = fmm.fmm_ref_gemm_fp64(A, B)
         errs = {}
