@@ -486,6 +486,72 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                     __syncwarp();
                     if (lane == 0) release_acc(0);
                     bphase ^= 1u;
+                } else if (C::DUMP) {
+                    // ---- output-warp kernel (block 32, 64 columns per warp).  The accumulators are read with the
+                    // 16-lane load shape: a thread owns four rows (lane/4 + 8k) x sixteen columns (8j + 2(lane%4), +1)
+                    // instead of one row x 64 columns, so it needs 16 B-side scales per K block instead of 64 (a
+                    // broadcast 16-byte shared-memory load returns 512 bytes to the register file; at one per four
+                    // elements those loads were a quarter of the promotion) and four A-side scales instead of one.
+                    static_assert(!C::DUMP || (C::CW == 64 && C::KB_PER_STAGE == 4 && C::GPB == 2), "output-warp kernel shape");
+#pragma unroll
+                    for (int i = 0; i < C::CW / 2; ++i) acc2[i] = 0ull;         // acc2[k * 8 + j]: row slot k, column group j
+                    const float4* sa_rows = reinterpret_cast<const float4*>(
+                        reinterpret_cast<const float*>(p.sa + (long long)t * p.sa_term) + (long long)(row_in_leaf + (lane >> 2)) * nkb);
+                    const long long row_step = 2ll * nkb;                       // eight rows further, in float4 units
+                    const uint32_t sb_lane = base + C::OFF_SB + (h * C::CW + 2 * (lane & 3)) * 4;
+                    for (int ks = 0; ks < kstages && ok; ++ks) {
+                        // the four K blocks of this stage for the thread's four rows; issued before the waits below,
+                        // which cover the load latency (a second set in flight would cost 16 more registers)
+                        float4 sa4[4];
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) sa4[k] = __ldg(sa_rows + k * row_step + ks);
+                        if (!mbar_wait_warp(bar_sfull(ss), sphase, ctl, 302)) { ok = false; break; }
+                        const uint32_t sbs32 = sb_lane + ss * C::SB_STAGE_BYTES;
+#pragma unroll
+                        for (int g0 = 0; g0 < C::KB_PER_STAGE; g0 += C::GPB) {
+                            const long long tw = TCLK();
+                            if (!mbar_wait_warp(bar_tfull(buf), bphase, ctl, 303)) { ok = false; break; }
+                            TADD(3, tw);
+                            tc_fence_after();
+#pragma unroll
+                            for (int gi = 0; gi < C::GPB; ++gi) {
+                                const int g = g0 + gi;
+                                const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (buf * C::GPB + gi) * BN + h * C::CW;
+#pragma unroll
+                                for (int c = 0; c < 2; ++c) {            // two halves of 32 columns
+                                    uint32_t lo[16], hi[16];
+                                    tmem_ld_16x256b_x4(taddr + c * 32, lo);                       // rows lane/4, lane/4 + 8
+                                    tmem_ld_16x256b_x4(taddr + c * 32 + (16u << 16), hi);         // rows lane/4 + 16, lane/4 + 24
+                                    unsigned long long sb2[4];
+#pragma unroll
+                                    for (int j = 0; j < 4; ++j) sb2[j] = lds64(sbs32 + (g * BN + c * 32 + 8 * j) * 4);
+                                    tmem_ld_wait();
+                                    if (gi + 1 == C::GPB && c == 1) {
+                                        // the last chunk is in registers: hand the TMEM buffers back before the arithmetic
+                                        tc_fence_before();
+                                        __syncwarp();
+                                        if (lane == 0) release_acc(buf);
+                                    }
+#pragma unroll
+                                    for (int k = 0; k < 4; ++k) {
+                                        const float sak = (g == 0) ? sa4[k].x : (g == 1) ? sa4[k].y : (g == 2) ? sa4[k].z : sa4[k].w;
+                                        const unsigned long long sa2 = pack2(sak, sak);
+                                        const uint32_t* src = (k < 2) ? lo : hi;
+#pragma unroll
+                                        for (int j = 0; j < 4; ++j) {
+                                            const uint32_t* tp = src + 4 * j + 2 * (k & 1);
+                                            acc2[k * 8 + c * 4 + j] = fma2(pack2u(tp[0], tp[1]), mul2(sa2, sb2[j]), acc2[k * 8 + c * 4 + j]);
+                                        }
+                                    }
+                                }
+                            }
+                            if (++buf == C::ACC_BUFS) { buf = 0; bphase ^= 1u; }
+                        }
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(bar_sempty(ss));
+                        if (++ss == C::SB_STAGES) { ss = 0; sphase ^= 1u; }
+                    }
+                    if (!ok) break;
                 } else {
 #pragma unroll
                     for (int i = 0; i < C::CW / 2; ++i) acc2[i] = 0ull;
@@ -579,16 +645,17 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                     const long long t_dump = TCLK();
                     if (!mbar_wait_warp(bar_dempty, dphase ^ 1u, ctl, 304)) { ok = false; break; }
                     dphase ^= 1u;
-                    uint8_t* dptr = base_ptr + C::OFF_DUMP + (q * (BN / 32) + h * (C::CW / 32)) * 4096 + lane * 128;
+                    // thread: rows lane/4 + 8k of the warp's 32-row chunk, column pairs 8j + 2(lane%4) of its 64 columns
+                    const uint32_t dchunk = base + C::OFF_DUMP + (q * (BN / 32) + h * (C::CW / 32)) * 4096 + (lane & 1) * 8;
 #pragma unroll
-                    for (int c = 0; c < C::CW / 32; ++c)
+                    for (int k = 0; k < 4; ++k) {
+                        const int rr = (lane >> 2) + 8 * k;
 #pragma unroll
-                        for (int i4 = 0; i4 < 8; ++i4) {
-                            float4 v;
-                            unpack2(acc2[c * 16 + i4 * 2], v.x, v.y);
-                            unpack2(acc2[c * 16 + i4 * 2 + 1], v.z, v.w);
-                            *reinterpret_cast<float4*>(dptr + c * 4096 + ((i4 ^ (lane & 7)) << 4)) = v;
+                        for (int j = 0; j < 8; ++j) {
+                            const int pc = 2 * (j & 3) + ((lane & 3) >> 1);        // 16-byte piece of the 128-byte row
+                            sts64(dchunk + (j >> 2) * 4096 + rr * 128 + ((pc ^ (rr & 7)) << 4), acc2[k * 8 + j]);
                         }
+                    }
                     __syncwarp();
                     if (lane == 0) mbar_arrive(bar_dfull);
                     TADD(4, t_dump);
