@@ -497,7 +497,7 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                     for (int i = 0; i < C::CW / 2; ++i) acc2[i] = 0ull;         // acc2[k * 8 + j]: row slot k, column group j
                     const float4* sa_rows = reinterpret_cast<const float4*>(
                         reinterpret_cast<const float*>(p.sa + (long long)t * p.sa_term) + (long long)(row_in_leaf + (lane >> 2)) * nkb);
-                    const long long row_step = 2ll * nkb;                       // eight rows further, in float4 units
+                    const int row_step = 2 * nkb;                               // eight rows further, in float4 units
                     const uint32_t sb_lane = base + C::OFF_SB + (h * C::CW + 2 * (lane & 3)) * 4;
                     for (int ks = 0; ks < kstages && ok; ++ks) {
                         // the four K blocks of this stage for the thread's four rows; issued before the waits below,
