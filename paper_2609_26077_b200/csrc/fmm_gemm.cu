@@ -38,7 +38,7 @@ constexpr int MODE_FP32_SB_TILE = 2;
 // a finished product to it through a shared-memory copy of the (unweighted) accumulators and go straight on with
 // the next term; the W-weighted stores / add-reductions then overlap the next term's promotion instead of stalling
 // it.  The output warp needs a fixed time per term, so this pays only when a term has many K stages (measured
-// cross-over between 16 and 32 stages of 128 k); the dispatcher picks the mode per launch.
+// cross-over near 16 stages of 128 k); the dispatcher picks the mode per launch.
 constexpr int MODE_FP32_OUT_WARP = 3;
 
 constexpr int BM = 128;                 // rows per CTA
@@ -62,6 +62,9 @@ struct Cfg {
     // staging space for more pipeline stages.
     static constexpr int STAGING_BUFS = (MX && NCTA == 2) ? 1 : 2;
     static constexpr bool DUMP = (MODE == MODE_FP32_OUT_WARP);
+    // FP32 scales, block 32: the promoting warps read the accumulators with the 16-lane load shape, four rows x
+    // sixteen columns per thread (see the promotion loop)
+    static constexpr bool ROWS4 = !MX && BK / BLK == 4 && BN == 128 && MODE != MODE_FP32_SB_TILE;
     static_assert(!DUMP || (BN == 128 && BK / BLK == 4), "output-warp mode: 128-column tiles, block 32");
     static constexpr int STAGES = (MX && NCTA == 2) ? 6 : ((A_BYTES + B_BYTES) > 40000 || DUMP ? 3 : 4);
     // DUMP (output-warp mode): shared-memory copy of a finished product, BM x BN fp32
@@ -486,13 +489,14 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                     __syncwarp();
                     if (lane == 0) release_acc(0);
                     bphase ^= 1u;
-                } else if (C::DUMP) {
-                    // ---- output-warp kernel (block 32, 64 columns per warp).  The accumulators are read with the
+                } else if (C::ROWS4) {
+                    // ---- block 32, 64 columns per warp.  The accumulators are read with the
                     // 16-lane load shape: a thread owns four rows (lane/4 + 8k) x sixteen columns (8j + 2(lane%4), +1)
                     // instead of one row x 64 columns, so it needs 16 B-side scales per K block instead of 64 (a
                     // broadcast 16-byte shared-memory load returns 512 bytes to the register file; at one per four
                     // elements those loads were a quarter of the promotion) and four A-side scales instead of one.
-                    static_assert(!C::DUMP || (C::CW == 64 && C::KB_PER_STAGE == 4 && C::GPB == 2), "output-warp kernel shape");
+                    static_assert(!C::ROWS4 || (C::CW == 64 && C::KB_PER_STAGE == 4 && C::GPB == 2), "block-32 kernel shape");
+                    static_assert(!C::DUMP || C::ROWS4, "the output warp expects the four-row register layout");
 #pragma unroll
                     for (int i = 0; i < C::CW / 2; ++i) acc2[i] = 0ull;         // acc2[k * 8 + j]: row slot k, column group j
                     const float4* sa_rows = reinterpret_cast<const float4*>(
@@ -684,6 +688,20 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                         // one row of the chunk per lane; 16-byte pieces permuted as the tensor map's swizzle expects
                         uint8_t* dst = stg_ptr + b * C::STAGING_BYTES + lane * (C::CH * 4);
                         const int swz = (C::CH == 32) ? (lane & 7) : ((lane >> 1) & 3);
+                        if (C::ROWS4) {
+                            // four-row layout: rows lane/4 + 8k, column pairs 8j + 2(lane%4) of this 32-column chunk
+                            const uint32_t sdst = stg + b * C::STAGING_BYTES + (lane & 1) * 8;
+                            const unsigned long long w2 = pack2(ent.w, ent.w);
+#pragma unroll
+                            for (int k = 0; k < 4; ++k) {
+                                const int rr = (lane >> 2) + 8 * k;
+#pragma unroll
+                                for (int j = 0; j < 4; ++j) {
+                                    const int pc = 2 * j + ((lane & 3) >> 1);
+                                    sts64(sdst + rr * 128 + ((pc ^ (rr & 7)) << 4), mul2(acc2[k * 8 + c * 4 + j], w2));
+                                }
+                            }
+                        } else
 #pragma unroll
                         for (int i4 = 0; i4 < C::CH / 4; ++i4) {
                             float4 v;
@@ -857,7 +875,7 @@ fmm_status_t launch_shape(const GemmParams& g, cudaStream_t st)
             if ((g.m % 256) == 0 && (g.n % 256) == 0) return launch<256, MODE, BLK, 2>(g, st);
         }
         if constexpr (BLK == 32 && MODE == FMM_SCALE_FP32_AMAX_DIV_448) {
-            if (g.k / BK >= 24) {           // long terms: post-addition by the output warp
+            if (g.k / BK >= 16) {           // long terms: post-addition by the output warp
                 if ((g.m % 256) == 0) return launch<128, MODE_FP32_OUT_WARP, BLK, 2>(g, st);
                 return launch<128, MODE_FP32_OUT_WARP, BLK, 1>(g, st);
             }
