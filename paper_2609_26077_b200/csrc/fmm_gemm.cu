@@ -62,9 +62,10 @@ struct Cfg {
     // staging space for more pipeline stages.
     static constexpr int STAGING_BUFS = (MX && NCTA == 2) ? 1 : 2;
     static constexpr bool DUMP = (MODE == MODE_FP32_OUT_WARP);
-    // FP32 scales, block 32: the promoting warps read the accumulators with the 16-lane load shape, four rows x
-    // sixteen columns per thread (see the promotion loop)
-    static constexpr bool ROWS4 = !MX && BK / BLK == 4 && BN == 128 && MODE != MODE_FP32_SB_TILE;
+    // FP32 scales per column: the promoting warps read the accumulators with the 16-lane load shape, four rows x
+    // CW/4 columns per thread (see the promotion loop).  The weight-tile mode has no per-column scale loads to
+    // save and is faster with one row per thread.
+    static constexpr bool ROWS4 = !MX && MODE != MODE_FP32_SB_TILE;
     static_assert(!DUMP || (BN == 128 && BK / BLK == 4), "output-warp mode: 128-column tiles, block 32");
     static constexpr int STAGES = (MX && NCTA == 2) ? 6 : ((A_BYTES + B_BYTES) > 40000 || DUMP ? 3 : 4);
     // DUMP (output-warp mode): shared-memory copy of a finished product, BM x BN fp32
@@ -490,25 +491,34 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                     if (lane == 0) release_acc(0);
                     bphase ^= 1u;
                 } else if (C::ROWS4) {
-                    // ---- block 32, 64 columns per warp.  The accumulators are read with the
-                    // 16-lane load shape: a thread owns four rows (lane/4 + 8k) x sixteen columns (8j + 2(lane%4), +1)
-                    // instead of one row x 64 columns, so it needs 16 B-side scales per K block instead of 64 (a
+                    // ---- per-column fp32 scales.  The accumulators are read with the
+                    // 16-lane load shape: a thread owns four rows (lane/4 + 8k) x CW/4 columns (8j + 2(lane%4), +1)
+                    // instead of one row x CW columns, so it needs CW/4 B-side scales per K block instead of CW (a
                     // broadcast 16-byte shared-memory load returns 512 bytes to the register file; at one per four
                     // elements those loads were a quarter of the promotion) and four A-side scales instead of one.
-                    static_assert(!C::ROWS4 || (C::CW == 64 && C::KB_PER_STAGE == 4 && C::GPB == 2), "block-32 kernel shape");
+                    static_assert(!C::ROWS4 || C::KB_PER_STAGE == 4 || C::KB_PER_STAGE == 1, "block 32 or 128");
                     static_assert(!C::DUMP || C::ROWS4, "the output warp expects the four-row register layout");
 #pragma unroll
-                    for (int i = 0; i < C::CW / 2; ++i) acc2[i] = 0ull;         // acc2[k * 8 + j]: row slot k, column group j
-                    const float4* sa_rows = reinterpret_cast<const float4*>(
-                        reinterpret_cast<const float*>(p.sa + (long long)t * p.sa_term) + (long long)(row_in_leaf + (lane >> 2)) * nkb);
-                    const int row_step = 2 * nkb;                               // eight rows further, in float4 units
+                    for (int i = 0; i < C::CW / 2; ++i) acc2[i] = 0ull;         // acc2[k * (CW/8) + j]: row slot k, column group j
+                    constexpr int JG = C::CW / 8;                               // column groups of eight per warp
+                    constexpr int KB = C::KB_PER_STAGE;
+                    const float* sa_rows = reinterpret_cast<const float*>(p.sa + (long long)t * p.sa_term) +
+                                           (long long)(row_in_leaf + (lane >> 2)) * nkb;
+                    const int row_step = 8 * nkb;                               // eight rows further
                     const uint32_t sb_lane = base + C::OFF_SB + (h * C::CW + 2 * (lane & 3)) * 4;
                     for (int ks = 0; ks < kstages && ok; ++ks) {
                         // the four K blocks of this stage for the thread's four rows; issued before the waits below,
                         // which cover the load latency (a second set in flight would cost 16 more registers)
-                        float4 sa4[4];
+                        float sa4[4][KB];
 #pragma unroll
-                        for (int k = 0; k < 4; ++k) sa4[k] = __ldg(sa_rows + k * row_step + ks);
+                        for (int k = 0; k < 4; ++k) {
+                            if constexpr (KB == 4) {
+                                const float4 v4 = __ldg(reinterpret_cast<const float4*>(sa_rows + k * row_step) + ks);
+                                sa4[k][0] = v4.x; sa4[k][1] = v4.y; sa4[k][2] = v4.z; sa4[k][3] = v4.w;
+                            } else {
+                                sa4[k][0] = __ldg(sa_rows + (k * row_step + ks));
+                            }
+                        }
                         if (!mbar_wait_warp(bar_sfull(ss), sphase, ctl, 302)) { ok = false; break; }
                         const uint32_t sbs32 = sb_lane + ss * C::SB_STAGE_BYTES;
 #pragma unroll
@@ -522,15 +532,20 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                                 const int g = g0 + gi;
                                 const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (buf * C::GPB + gi) * BN + h * C::CW;
 #pragma unroll
-                                for (int c = 0; c < 2; ++c) {            // two halves of 32 columns
+                                float sbt = 1.0f;
+                                if (MODE == MODE_FP32_SB_TILE) sbt = *reinterpret_cast<const float*>(base_ptr + C::OFF_SB + ss * C::SB_STAGE_BYTES + (g * BN + h * C::CW) * 4);
+#pragma unroll
+                                for (int c = 0; c < C::CW / 32; ++c) {   // chunks of 32 columns
                                     uint32_t lo[16], hi[16];
                                     tmem_ld_16x256b_x4(taddr + c * 32, lo);                       // rows lane/4, lane/4 + 8
                                     tmem_ld_16x256b_x4(taddr + c * 32 + (16u << 16), hi);         // rows lane/4 + 16, lane/4 + 24
                                     unsigned long long sb2[4];
+                                    if (MODE != MODE_FP32_SB_TILE) {
 #pragma unroll
-                                    for (int j = 0; j < 4; ++j) sb2[j] = lds64(sbs32 + (g * BN + c * 32 + 8 * j) * 4);
+                                        for (int j = 0; j < 4; ++j) sb2[j] = lds64(sbs32 + (g * BN + c * 32 + 8 * j) * 4);
+                                    }
                                     tmem_ld_wait();
-                                    if (gi + 1 == C::GPB && c == 1) {
+                                    if (gi + 1 == C::GPB && c + 1 == C::CW / 32) {
                                         // the last chunk is in registers: hand the TMEM buffers back before the arithmetic
                                         tc_fence_before();
                                         __syncwarp();
@@ -538,13 +553,14 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                                     }
 #pragma unroll
                                     for (int k = 0; k < 4; ++k) {
-                                        const float sak = (g == 0) ? sa4[k].x : (g == 1) ? sa4[k].y : (g == 2) ? sa4[k].z : sa4[k].w;
+                                        const float sak = sa4[k][g] * sbt;       // tile mode: sA * sB_tile; else sbt = 1 (folded away)
                                         const unsigned long long sa2 = pack2(sak, sak);
                                         const uint32_t* src = (k < 2) ? lo : hi;
 #pragma unroll
                                         for (int j = 0; j < 4; ++j) {
                                             const uint32_t* tp = src + 4 * j + 2 * (k & 1);
-                                            acc2[k * 8 + c * 4 + j] = fma2(pack2u(tp[0], tp[1]), mul2(sa2, sb2[j]), acc2[k * 8 + c * 4 + j]);
+                                            const unsigned long long s2 = (MODE == MODE_FP32_SB_TILE) ? sa2 : mul2(sa2, sb2[j]);
+                                            acc2[k * JG + c * 4 + j] = fma2(pack2u(tp[0], tp[1]), s2, acc2[k * JG + c * 4 + j]);
                                         }
                                     }
                                 }
@@ -698,7 +714,7 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
 #pragma unroll
                                 for (int j = 0; j < 4; ++j) {
                                     const int pc = 2 * j + ((lane & 3) >> 1);
-                                    sts64(sdst + rr * 128 + ((pc ^ (rr & 7)) << 4), mul2(acc2[k * 8 + c * 4 + j], w2));
+                                    sts64(sdst + rr * 128 + ((pc ^ (rr & 7)) << 4), mul2(acc2[k * (C::CW / 8) + c * 4 + j], w2));
                                 }
                             }
                         } else

@@ -39,7 +39,7 @@ CASES = [
     ("strassen", 1, (5120, 512, 4096), 32, "ue8m0", "gaussian"),
     ("phi_optimal", 1, (4864, 256, 4096), 32, "ue8m0", "uniform"),
     ("strassen", 1, (5120, 512, 4096), 128, "fp32", "gaussian"),
-    # 24 or more K stages per term: fp32 / block-32 products take the kernel variant with the output warp
+    # 16 or more K stages per term: fp32 / block-32 products take the kernel variant with the output warp
     ("cubic", 0, (256, 3072, 384), 32, "fp32", "gaussian"),
     ("phi_optimal", 1, (512, 6144, 768), 32, "fp32", "llm"),
     ("winograd", 1, (768, 8192, 256), 32, "fp32", "uniform"),
