@@ -616,20 +616,6 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
 #pragma unroll
                                 for (int c = 0; c < C::CW / 32; ++c) {
                                     tmem_ld32(taddr + c * 32, tmp);      // a TMEM load round trip is a few tens of cycles
-                                    // the scale products do not depend on the accumulator: they are formed while the
-                                    // TMEM load is in flight (the wait below is a barrier for the compiler's scheduler)
-                                    // (measured: helps with one promotion per 128 k, hurts with one per 32 k, where the
-                                    // compiler's own interleaving of the two granules is better)
-                                    constexpr bool HOIST = (BLK == 128) && MODE != MODE_FP32_SB_TILE;
-                                    unsigned long long sp[HOIST ? 16 : 1];
-                                    if (HOIST) {
-#pragma unroll
-                                        for (int i = 0; i < 8; ++i) {
-                                            const ulonglong2 s4 = sbg[c * 8 + i];        // four column scales
-                                            sp[HOIST ? 2 * i : 0] = mul2(sa2, s4.x);
-                                            sp[HOIST ? 2 * i + 1 : 0] = mul2(sa2, s4.y);
-                                        }
-                                    }
                                     tmem_ld_wait();
                                     if (gi + 1 == C::GPB && c + 1 == C::CW / 32) {
                                         // the last chunk is in registers: hand the TMEM buffers back before the arithmetic
@@ -641,8 +627,7 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                                     for (int i = 0; i < 8; ++i) {
                                         const uint32_t* tp = tmp + 4 * i;
                                         unsigned long long s01 = sa2, s23 = sa2;        // tile mode: sA * sB_tile
-                                        if (HOIST) { s01 = sp[HOIST ? 2 * i : 0]; s23 = sp[HOIST ? 2 * i + 1 : 0]; }
-                                        else if (MODE != MODE_FP32_SB_TILE) {
+                                        if (MODE != MODE_FP32_SB_TILE) {
                                             const ulonglong2 s4 = sbg[c * 8 + i];        // four column scales
                                             s01 = mul2(sa2, s4.x); s23 = mul2(sa2, s4.y);
                                         }
