@@ -126,10 +126,12 @@ def test_paper_emulated_error_figures_blk128_signed_uniform():
     # Table E.1 row <2,2,2>: blk128, signed-uniform operands, block edge 256 (n = 512), one level,
     # eight paired samples: e_lib/e_cub = 2.4486 at e_lib = 0.0874 gives e_cubic = 0.03569;
     # re-based (Phi-optimal) / cubic = 1.7190.  App. D: s_q ~ 0.0253 predicts e_cubic ~ s_q sqrt 2.
+    from golden_values import figures
+    g = figures()                    # tests/golden/printed_figures.json
     e = _mean_errors(Wl.uniform, 512, 128, 1, range(8))
-    assert e["cubic"] == pytest.approx(0.0874 / 2.4486, rel=0.02)
-    assert e["cubic"] == pytest.approx(0.0253 * math.sqrt(2), rel=0.02)
-    assert e["phi_optimal"] / e["cubic"] == pytest.approx(1.7190, rel=0.02)
+    assert e["cubic"] == pytest.approx(g["e_lib_222"] / g["e_lib_over_e_cubic_222"], rel=0.02)
+    assert e["cubic"] == pytest.approx(g["s_q"] * math.sqrt(2), rel=0.02)
+    assert e["phi_optimal"] / e["cubic"] == pytest.approx(g["rebased_over_cubic_222"], rel=0.02)
     # Phi-predicted ordering and magnitudes (Sec. 3): 5/3 < 2 < sqrt 7
     assert e["strassen"] / e["cubic"] == pytest.approx(2.0, rel=0.04)
     assert e["winograd"] / e["cubic"] == pytest.approx(math.sqrt(7), rel=0.04)

@@ -36,9 +36,14 @@ def test_phi_values_exact():
 
 def test_gamma_values():
     # Table E.2 and App. C
-    assert R.gamma(*R.strassen()) == pytest.approx(14.8284, abs=5e-5)
-    assert R.gamma(*R.winograd()) == pytest.approx(17.8530, abs=5e-5)
-    assert R.gamma(*R.phi_optimal()) == pytest.approx(12.066031431780, abs=1e-11)
+    from golden_values import figures, panel
+    tab = panel()                    # Table E.2 as printed (tests/golden/table_e2_panel.tsv)
+    assert R.gamma(*R.strassen()) == pytest.approx(tab["strassen_classic"][2], abs=5e-5)
+    assert R.gamma(*R.winograd()) == pytest.approx(tab["winograd_form"][2], abs=5e-5)
+    assert R.gamma(*R.phi_optimal()) == pytest.approx(tab["dps_acc"][2], abs=5e-5)
+    assert R.gamma(*R.phi_optimal()) == pytest.approx(figures()["gamma_optimal_exact"], abs=1e-11)
+    assert float(R.phi(*R.strassen()).a) == tab["strassen_classic"][1] and float(R.phi(*R.winograd()).a) == tab["winograd_form"][1]
+    assert float(R.phi(*R.phi_optimal()).a) == pytest.approx(tab["dps_acc"][1], abs=5e-5)
     assert R.gamma(*R.phi_optimal()) == pytest.approx(2 * math.sqrt(2) + 16 / math.sqrt(3), abs=1e-12)
 
 

@@ -100,15 +100,22 @@ def test_gamma_values_against_the_printed_panel():
     # Strassen, 17.8530 for the Winograd form, and, for the twelve Phi = 24 arms, 12.4549 / 12.4791 (six arms)
     # and values between 12.4658 and 12.4683 (six arms).  The artifact's coordinate frame is not printed, so
     # arm labels cannot be matched one to one; the two families of values can.
+    from golden_values import panel
+    tab = panel()                    # tests/golden/table_e2_panel.tsv
     g = lambda n: R.gamma(*[[[float(x) for x in r] for r in M] for M in P.get64(n)])
-    assert round(g("phi_optimal"), 4) == 12.0660
-    assert round(g("strassen"), 4) == 14.8284
-    assert round(g("winograd"), 4) == 17.8530
+    assert round(g("phi_optimal"), 4) == tab["dps_acc"][2]
+    assert round(g("strassen"), 4) == tab["strassen_classic"][2]
+    assert round(g("winograd"), 4) == tab["winograd_form"][2]
+    printed = sorted(v[2] for k, v in tab.items() if v[0] == "P")
+    assert all(v[1] == 24.0 for v in tab.values() if v[0] == "P") and len(printed) == 12
+    # the printed values fall into two families: three arms each at the two extremes, six in between
+    lo, hi = printed[0], printed[-1]
+    assert printed[:3] == [lo] * 3 and printed[-3:] == [hi] * 3
     extreme = sorted(round(g(n), 4) for n in P.PERTURBATIONS if "_diag_" in n)
-    assert extreme == [12.4549] * 3 + [12.4791] * 3
+    assert extreme == [lo] * 3 + [hi] * 3
     for n in P.PERTURBATIONS:
         if "_shear_" in n:
-            assert 12.4658 - 0.0015 < g(n) < 12.4683 + 0.0015
+            assert printed[3] - 0.0015 < g(n) < printed[8] + 0.0015
         assert abs(g(n) - g(n + "_rb")) < 1e-12       # Gamma does not see the gauge
 
 
