@@ -531,7 +531,6 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                             for (int gi = 0; gi < C::GPB; ++gi) {
                                 const int g = g0 + gi;
                                 const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (buf * C::GPB + gi) * BN + h * C::CW;
-#pragma unroll
                                 float sbt = 1.0f;
                                 if (MODE == MODE_FP32_SB_TILE) sbt = *reinterpret_cast<const float*>(base_ptr + C::OFF_SB + ss * C::SB_STAGE_BYTES + (g * BN + h * C::CW) * 4);
 #pragma unroll
