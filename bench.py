@@ -215,21 +215,46 @@ def run_ours(args):
     clocks = sampler.stop()
     status = plan.device_status()
 
-    # ---- end to end: host buffers, copies inside the timed region
+    # ---- end to end: the library's host-operand call, host buffers in pinned memory, copies inside the timed region.
+    # Two streams, each with its own device workspace and its own result buffer, take alternate steps, so that one
+    # step's upload overlaps the previous step's product and download (every step still moves all of its inputs
+    # and its result across the host link inside the timed region).
     Ah = torch.empty(M, K, dtype=torch.float32, pin_memory=True)
     Bh = torch.empty(K, N, dtype=torch.float32, pin_memory=True)
-    Ch = torch.empty(M, N, dtype=torch.float32, pin_memory=True)
     Ah.copy_(A); Bh.copy_(B)
-    Ad, Bd = torch.empty_like(A), torch.empty_like(B)
+    lanes = 2
+    e2e_streams = [torch.cuda.Stream() for _ in range(lanes)]
+    e2e_ws = [plan.host_workspace(M, N, K) for _ in range(lanes)]
+    Ch = [torch.empty(M, N, dtype=torch.float32, pin_memory=True) for _ in range(lanes)]
+    e2e_count = [0]
 
     def e2e_step():
-        Ad.copy_(Ah, non_blocking=True)
-        Bd.copy_(Bh, non_blocking=True)
-        plan.matmul(Ad, Bd, out=C, workspace=ws)
-        Ch.copy_(C, non_blocking=True)
+        i = e2e_count[0] % lanes
+        e2e_count[0] += 1
+        plan.matmul_host(Ah, Bh, Ch[i], e2e_ws[i], stream=e2e_streams[i])
 
-    e2e_steps = max(3, min(K_steps, 10))
-    ms_e2e = time_steps(e2e_step, e2e_steps, 3)
+    def time_e2e(steps, warm):
+        cur = torch.cuda.current_stream()
+        for _ in range(warm):
+            e2e_step()
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        for st in e2e_streams:
+            st.wait_stream(cur)
+        e0.record(cur)
+        for st in e2e_streams:
+            st.wait_event(e0)
+        for _ in range(steps):
+            e2e_step()
+        for st in e2e_streams:
+            cur.wait_stream(st)
+        e1.record(cur)
+        barrier()
+        return reduce_max_ms(e0.elapsed_time(e1), dist, "cuda") / steps
+
+    e2e_steps = max(4, min(K_steps, 10))
+    ms_e2e = time_e2e(e2e_steps, 4)
+    e2e_ok = bool(torch.equal(Ch[0], Ch[1]) and torch.equal(Ch[0], C.cpu()))
 
     flop_eff = 2.0 * M * N * K
     value = replica_throughput(flop_eff, world, ms_step)
@@ -251,7 +276,9 @@ def run_ours(args):
         "clocks": clocks,
         "gpu_launches": launches_per_step * K_steps,
         "e2e": {"value": replica_throughput(flop_eff, world, ms_e2e), "unit": UNIT, "ms_per_step": ms_e2e,
-                "h2d_bytes_per_step": 4 * (M * K + K * N), "d2h_bytes_per_step": 4 * M * N, "steps": e2e_steps},
+                "h2d_bytes_per_step": 4 * (M * K + K * N), "d2h_bytes_per_step": 4 * M * N, "steps": e2e_steps,
+                "call": "fmm_matmul_host, 2 streams x own workspace (uploads overlap the other stream's product and download)",
+                "result_matches_device_path": e2e_ok},
         "phases": {"encode_ms": enc_ms, "multiply_ms": mul_ms,
                    "encode_hbm_frac": enc_bytes / (enc_ms * 1e-3) / 1e9 / hbm,
                    "encode_gbs": enc_bytes / (enc_ms * 1e-3) / 1e9,

@@ -107,6 +107,21 @@ fmm_status_t fmm_matmul(const fmm_plan_t* plan, const float* A, const float* B, 
                         int64_t M, int64_t N, int64_t K, void* workspace, size_t workspace_bytes,
                         void* cuda_stream);
 
+/* The same product with HOST operands: uploads A and B, runs fmm_matmul on the device copies, downloads C.
+ *   A host, M x K fp32;  B host, K x N fp32;  C host, M x N fp32, overwritten.  Page-locked (pinned) host
+ *   memory makes the three copies asynchronous; pageable memory works but the copies then block the caller.
+ *   workspace dev, 1024-byte aligned, at least fmm_host_workspace_bytes() bytes, caller-owned: the product's
+ *   workspace followed by device staging for A, B and C.
+ * Everything is enqueued on cuda_stream in order (upload A, upload B, product, download C) and nothing is
+ * synchronised: C is valid once the stream has drained.  Calls on different streams with different workspaces
+ * overlap one call's uploads with another's product and download (the links are full duplex); that is the
+ * intended use for a sequence of products.  Errors as fmm_matmul. */
+fmm_status_t fmm_host_workspace_bytes(const fmm_plan_t* plan, int64_t M, int64_t N, int64_t K,
+                                      size_t* bytes);
+fmm_status_t fmm_matmul_host(const fmm_plan_t* plan, const float* A, const float* B, float* C,
+                             int64_t M, int64_t N, int64_t K, void* workspace, size_t workspace_bytes,
+                             void* cuda_stream);
+
 /* Steps 1-2 only (pre-addition + quantization of both sides) into the workspace. */
 fmm_status_t fmm_encode_only(const fmm_plan_t* plan, const float* A, const float* B,
                              int64_t M, int64_t N, int64_t K, void* workspace,

@@ -431,6 +431,46 @@ fmm_status_t fmm_matmul(const fmm_plan_t* cplan, const float* A, const float* B,
     return multiply(plan, L, static_cast<char*>(ws), C, M, N, st);
 }
 
+// Host-operand variant: [product workspace | A | B | C] in the caller's device buffer, 1024-byte aligned parts.
+static size_t host_align(size_t x) { return (x + 1023) & ~(size_t)1023; }
+
+fmm_status_t fmm_host_workspace_bytes(const fmm_plan_t* plan, int64_t M, int64_t N, int64_t K, size_t* bytes)
+{
+    size_t ws = 0;
+    fmm_status_t s = fmm_workspace_bytes(plan, M, N, K, &ws);
+    if (s != FMM_OK) return s;
+    *bytes = host_align(ws) + host_align((size_t)M * K * 4) + host_align((size_t)K * N * 4) + host_align((size_t)M * N * 4);
+    return FMM_OK;
+}
+
+fmm_status_t fmm_matmul_host(const fmm_plan_t* plan, const float* A, const float* B, float* C,
+                             int64_t M, int64_t N, int64_t K, void* ws, size_t ws_bytes, void* stream)
+{
+    if (!plan || !A || !B || !C) return FMM_ERR_INVALID_ARG;
+    size_t need = 0, inner = 0;
+    fmm_status_t s = fmm_host_workspace_bytes(plan, M, N, K, &need);
+    if (s != FMM_OK) return s;
+    if (!ws || ((uintptr_t)ws & 1023) || ws_bytes < need) return FMM_ERR_WORKSPACE;
+    fmm_workspace_bytes(plan, M, N, K, &inner);
+    char* base = static_cast<char*>(ws);
+    float* dA = reinterpret_cast<float*>(base + host_align(inner));
+    float* dB = reinterpret_cast<float*>(reinterpret_cast<char*>(dA) + host_align((size_t)M * K * 4));
+    float* dC = reinterpret_cast<float*>(reinterpret_cast<char*>(dB) + host_align((size_t)K * N * 4));
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    if (cudaMemcpyAsync(dA, A, (size_t)M * K * 4, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+        cudaMemcpyAsync(dB, B, (size_t)K * N * 4, cudaMemcpyHostToDevice, st) != cudaSuccess) {
+        cudaGetLastError();
+        return FMM_ERR_CUDA;
+    }
+    s = fmm_matmul(plan, dA, dB, dC, M, N, K, ws, inner, stream);
+    if (s != FMM_OK) return s;
+    if (cudaMemcpyAsync(C, dC, (size_t)M * N * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess) {
+        cudaGetLastError();
+        return FMM_ERR_CUDA;
+    }
+    return FMM_OK;
+}
+
 fmm_status_t fmm_device_status(const fmm_plan_t* plan, int* code)
 {
     if (!plan || !code) return FMM_ERR_INVALID_ARG;

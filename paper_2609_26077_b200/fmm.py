@@ -16,7 +16,8 @@ STATUS_NAMES = ["FMM_OK", "FMM_ERR_INVALID_ARG", "FMM_ERR_SHAPE", "FMM_ERR_NOT_E
 SCALE_FP32, SCALE_UE8M0 = 0, 1
 SCALE_MODES = {"fp32": SCALE_FP32, "ue8m0": SCALE_UE8M0}
 
-EXPORTS = ["fmm_plan_create", "fmm_plan_destroy", "fmm_workspace_bytes", "fmm_matmul", "fmm_encode_only",
+EXPORTS = ["fmm_plan_create", "fmm_plan_destroy", "fmm_workspace_bytes", "fmm_matmul", "fmm_host_workspace_bytes",
+           "fmm_matmul_host", "fmm_encode_only",
            "fmm_multiply_only", "fmm_quantized_view", "fmm_ref_gemm_fp64", "fmm_error_stats",
            "fmm_error_stats_scratch_bytes", "fmm_error_stats_noalloc", "fmm_error_stats_noalloc_max_elements",
            "fmm_device_status", "fmm_device_status_clear", "fmm_selftest_bounded_wait", "fmm_phi_gamma", "fmm_brent_residual",
@@ -155,6 +156,29 @@ class Plan:
         ws = workspace if workspace is not None else self.workspace(M, N, K, A.device)
         _check(lib().fmm_matmul(self._h, _dev_ptr(A), _dev_ptr(B), _dev_ptr(out), C.c_int64(M), C.c_int64(N),
                                 C.c_int64(K), _dev_ptr(ws), C.c_size_t(ws.numel()), _stream_ptr(stream)), "fmm_matmul")
+        return out
+
+    def host_workspace(self, M, N, K, device="cuda"):
+        """Device buffer for matmul_host: fmm_host_workspace_bytes, 1024-byte aligned (a fresh tensor per call)."""
+        import torch
+        need = C.c_size_t()
+        _check(lib().fmm_host_workspace_bytes(self._h, C.c_int64(M), C.c_int64(N), C.c_int64(K), C.byref(need)),
+               "fmm_host_workspace_bytes")
+        buf = torch.empty(need.value + 1024, dtype=torch.uint8, device=device)
+        off = (-buf.data_ptr()) % 1024
+        return buf[off:off + need.value]
+
+    def matmul_host(self, A, B, out, workspace, stream=None):
+        """fmm_matmul_host: host operands (pinned for asynchronous copies), C written to the host tensor `out`."""
+        import torch
+        M, K = A.shape
+        K2, N = B.shape
+        assert K == K2 and tuple(out.shape) == (M, N)
+        for t in (A, B, out):
+            assert t.dtype == torch.float32 and t.is_contiguous() and not t.is_cuda
+        _check(lib().fmm_matmul_host(self._h, C.c_void_p(A.data_ptr()), C.c_void_p(B.data_ptr()), C.c_void_p(out.data_ptr()),
+                                     C.c_int64(M), C.c_int64(N), C.c_int64(K), _dev_ptr(workspace),
+                                     C.c_size_t(workspace.numel()), _stream_ptr(stream)), "fmm_matmul_host")
         return out
 
     def encode_only(self, A, B, workspace=None, stream=None):

@@ -118,3 +118,48 @@ def test_matmul_can_be_captured_in_a_cuda_graph():
         torch.cuda.synchronize()
         assert torch.equal(out, eager)
         assert plan.device_status() == (0, 0)
+
+
+@pytest.mark.parametrize("pinned", [True, False])
+def test_host_operand_call_matches_the_device_call_bit_for_bit(pinned):
+    # fmm_matmul_host = upload, fmm_matmul, download: same kernels on the same bytes, so C is identical; two calls on two
+    # streams with their own workspaces may overlap and must not disturb each other
+    M, K, N = 512, 768, 256
+    A, B = Wl.gaussian(M, K, N, 9)
+    plan = make_plan("phi_optimal", 1, 32, "fp32")
+    want = plan.matmul(dev(A), dev(B)).cpu()
+    Ah, Bh = torch.from_numpy(A).clone(), torch.from_numpy(B).clone()
+    if pinned:
+        Ah, Bh = Ah.pin_memory(), Bh.pin_memory()
+    streams = [torch.cuda.Stream() for _ in range(2)]
+    wss = [plan.host_workspace(M, N, K) for _ in range(2)]
+    outs = [torch.full((M, N), float("nan")) for _ in range(2)]
+    if pinned:
+        outs = [o.pin_memory() for o in outs]
+    torch.cuda.synchronize()
+    for rep in range(2):
+        for i in range(2):
+            plan.matmul_host(Ah, Bh, outs[i], wss[i], stream=streams[i])
+    torch.cuda.synchronize()
+    assert plan.device_status() == (0, 0)
+    assert torch.equal(outs[0], want) and torch.equal(outs[1], want)
+
+
+def test_host_operand_call_rejects_bad_arguments():
+    plan = make_plan("strassen", 1, 32, "ue8m0")
+    lib = fmm.lib()
+    h = torch.zeros(256, 256)
+    ws = plan.host_workspace(256, 256, 256)
+    inner = plan.workspace_bytes(256, 256, 256)
+    assert ws.numel() >= inner + 3 * 256 * 256 * 4
+    p = lambda t: C.c_void_p(t.data_ptr())
+    call = lambda M, w, wb, A=h: lib.fmm_matmul_host(plan._h, p(A) if A is not None else None, p(h), p(h), C.c_int64(M),
+                                                     C.c_int64(256), C.c_int64(256), w, C.c_size_t(wb), None)
+    assert call(256, p(ws), ws.numel()) == 0
+    torch.cuda.synchronize()
+    assert call(192, p(ws), ws.numel()) == 2
+    assert call(256, p(ws), inner) == 4                 # room for the product's workspace only
+    assert call(256, None, ws.numel()) == 4
+    assert call(256, p(ws), ws.numel(), A=None) == 1
+    need = C.c_size_t()
+    assert lib.fmm_host_workspace_bytes(plan._h, C.c_int64(100), C.c_int64(256), C.c_int64(256), C.byref(need)) == 2
