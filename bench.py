@@ -139,6 +139,20 @@ def algorithmic_work(M, N, K, levels, rank, scale_bytes, blk):
     return flops, enc_bytes, gemm_bytes
 
 
+def combined_roofline_ms(M, N, K, levels, rank, mode, blk, fp8_peak_tflops, hbm_gbs):
+    """Combined roofline time of one pass: the product phase at the measured fp8 tensor peak - or, with fp32 scales, at
+    the CUDA-core bound of the per-block promotion if that is larger - plus the algorithmic HBM bytes at the measured
+    copy bandwidth (phases serialized)."""
+    scale_bytes = 1 if mode == "ue8m0" else 4
+    flops, enc_bytes, gemm_bytes = algorithmic_work(M, N, K, levels, rank, scale_bytes, blk)
+    t_main = flops / (fp8_peak_tflops * 1e12)
+    if mode != "ue8m0":
+        f = (rank / 8.0) ** levels if levels > 0 else 1.0
+        ops = 1.0 if "tile" in mode else 2.0        # weight tiles: the factor is formed once per row, one FMA per element
+        t_main = max(t_main, ops * M * N * (K / blk) * f / (148 * 128 * 1.965e9))
+    return (t_main + (enc_bytes + gemm_bytes) / (hbm_gbs * 1e9)) * 1e3
+
+
 def run_ours(args):
     import numpy as np
     import torch
@@ -330,8 +344,10 @@ def run_ours(args):
             p2 = make_plan(name, lv, blk, mode)
             w2 = p2.workspace(M, N, K)
             ms = time_steps(lambda: p2.matmul(A, B, out=C, workspace=w2), 5, 3)
+            t_roof = combined_roofline_ms(M, N, K, lv, p2.rank if lv > 0 else 8, mode, blk, fp8_peak, hbm)
             variants.append({"realization": name, "levels": lv, "block_k": blk, "scale_mode": mode,
-                             "ms_per_step": ms, "value": flop_eff / (ms * 1e-3) / 1e12})
+                             "ms_per_step": ms, "value": flop_eff / (ms * 1e-3) / 1e12,
+                             "combined_roofline_ms": t_roof, "combined_frac": t_roof / ms})
             p2.close()
         out["variants"] = variants
         # the paper's timing protocol (App. E.7): interleaved repetitions across realizations, median and a
