@@ -15,8 +15,9 @@ static __device__ __align__(256) double g_noalloc_partials[3 * 1024];
 
 namespace {
 
-constexpr int STAT_BLOCKS = 1024;     // also the number of slots of g_noalloc_partials
-constexpr int STAT_THREADS = 256;
+constexpr int STAT_BLOCKS = 592;      // 4 x 148 SMs, all resident at 512 threads; at most the 1024 slots of g_noalloc_partials
+constexpr int STAT_THREADS = 512;
+static_assert(STAT_BLOCKS <= 1024, "one scratch slot per reduction block");
 
 __device__ __forceinline__ void warp_reduce3(double& a, double& b, double& c)
 {
@@ -49,16 +50,27 @@ __global__ void __launch_bounds__(STAT_THREADS) error_partial_kernel(const float
 {
     __shared__ double sm[3 * (STAT_THREADS / 32)];
     double sd = 0.0, sr = 0.0, mx = 0.0;
-    // each thread takes pairs: one 8-byte load of C, one 16-byte load of Cref (count is even)
+    // each thread takes pairs: one 8-byte load of C, one 16-byte load of Cref (count is even); four pairs per
+    // trip with all loads issued first, so that every thread keeps 96 bytes in flight
     const int64_t pairs = count >> 1;
-    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < pairs; i += (int64_t)gridDim.x * blockDim.x) {
-        const float2 c = __ldcs(reinterpret_cast<const float2*>(C) + i);
-        const double2 r = __ldcs(reinterpret_cast<const double2*>(Cref) + i);
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    const float2* C2 = reinterpret_cast<const float2*>(C);
+    const double2* R2 = reinterpret_cast<const double2*>(Cref);
+    auto add = [&](float2 c, double2 r) {
         const double d0 = (double)c.x - r.x, d1 = (double)c.y - r.y;
         sd = fma(d0, d0, sd); sd = fma(d1, d1, sd);
         sr = fma(r.x, r.x, sr); sr = fma(r.y, r.y, sr);
         mx = fmax(mx, fmax(fabs(d0), fabs(d1)));
+    };
+    int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    for (; i + 3 * stride < pairs; i += 4 * stride) {
+        float2 c[4]; double2 r[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) { c[u] = __ldcs(C2 + i + u * stride); r[u] = __ldcs(R2 + i + u * stride); }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) add(c[u], r[u]);
     }
+    for (; i < pairs; i += stride) add(__ldcs(C2 + i), __ldcs(R2 + i));
     block_reduce3(sd, sr, mx, sm);
     if (threadIdx.x == 0) {
         partial[blockIdx.x * 3] = sd; partial[blockIdx.x * 3 + 1] = sr; partial[blockIdx.x * 3 + 2] = mx;
@@ -161,7 +173,7 @@ fmm_status_t fmm_ref_gemm_fp64(const float* A, const float* B, double* Cref, int
 // ---- variant of fmm_error_stats for callers that cannot allocate device memory ----------------
 namespace {
 constexpr int NOALLOC_MAX_DEVICES = 64;
-constexpr int64_t NOALLOC_MAX_ELEMS = (int64_t)1 << 28;    // 1024 scratch slots x at most 2^18 elements each
+constexpr int64_t NOALLOC_MAX_ELEMS = (int64_t)1 << 28;    // limit of the interface (2^18 elements per slot of the 1024-slot array)
 std::mutex g_noalloc_mutex;
 double* g_noalloc_ptr[NOALLOC_MAX_DEVICES] = {nullptr};
 
