@@ -541,8 +541,15 @@ __global__ void __launch_bounds__(256) decode_kernel(const DecodeParams p)
 #pragma unroll
         for (int q = 0; q < 4; ++q) acc[q] = make_float4(0.f, 0.f, 0.f, 0.f);
         const float* src = p.in + ((int64_t)b * p.R) * in_stride + (int64_t)i * p.cols + c * 4;
-        for (int r = 0; r < p.R; ++r) {
-            const float4 x = __ldcs(reinterpret_cast<const float4*>(src + r * in_stride));
+        // all R loads are issued before the first use (R x 16 bytes in flight per thread)
+        float4 xs[FMM_MAX_RANK];
+#pragma unroll
+        for (int r = 0; r < FMM_MAX_RANK; ++r)
+            if (r < p.R) xs[r] = __ldcs(reinterpret_cast<const float4*>(src + r * in_stride));
+#pragma unroll
+        for (int r = 0; r < FMM_MAX_RANK; ++r) {
+            if (r >= p.R) break;
+            const float4 x = xs[r];
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
                 const float w = p.W[r][q];
