@@ -97,7 +97,8 @@ fmm_status_t fmm_workspace_bytes(const fmm_plan_t* plan, int64_t M, int64_t N, i
 
 /* C = A * B through the plan's realization (whole hot path: pre-addition + quantization of both
  * sides, the R^levels block-scaled fp8 products on the tensor cores, post-addition into C).
- *   A dev, M x K fp32;  B dev, K x N fp32;  C dev, M x N fp32, overwritten.
+ *   A dev, M x K fp32;  B dev, K x N fp32;  C dev, M x N fp32, overwritten.  All three 16-byte aligned
+ *   (vector loads, tensor-map stores), else FMM_ERR_INVALID_ARG.
  *   Shape rule: with d = 2^levels, M/d and N/d must be multiples of 128 and K/d a multiple of 128
  *   (hence of block_k); otherwise FMM_ERR_SHAPE.
  *   workspace dev, 1024-byte aligned, at least fmm_workspace_bytes() bytes, caller-owned; its

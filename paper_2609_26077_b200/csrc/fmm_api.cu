@@ -76,6 +76,9 @@ void make_layout(const fmm_plan* plan, int64_t M, int64_t N, int64_t K, FmmLayou
     L->total = off;
 }
 
+// the kernels read the operands with 16-byte vector loads and write C through a tensor map
+bool aligned16(const void* p) { return ((uintptr_t)p & 15) == 0; }
+
 fmm_status_t check_ws(const fmm_plan* plan, int64_t M, int64_t N, int64_t K, void* ws, size_t ws_bytes,
                       FmmLayout* L)
 {
@@ -390,7 +393,7 @@ fmm_status_t fmm_quantized_view(const fmm_plan_t* plan, int64_t M, int64_t N, in
 fmm_status_t fmm_encode_only(const fmm_plan_t* cplan, const float* A, const float* B, int64_t M, int64_t N, int64_t K,
                              void* ws, size_t ws_bytes, void* stream)
 {
-    if (!cplan || !A || !B) return FMM_ERR_INVALID_ARG;
+    if (!cplan || !A || !B || !aligned16(A) || !aligned16(B)) return FMM_ERR_INVALID_ARG;
     fmm_plan* plan = const_cast<fmm_plan*>(cplan);
     FmmLayout L;
     fmm_status_t s = check_ws(plan, M, N, K, ws, ws_bytes, &L);
@@ -405,7 +408,7 @@ fmm_status_t fmm_encode_only(const fmm_plan_t* cplan, const float* A, const floa
 fmm_status_t fmm_multiply_only(const fmm_plan_t* cplan, float* C, int64_t M, int64_t N, int64_t K,
                                void* ws, size_t ws_bytes, void* stream)
 {
-    if (!cplan || !C) return FMM_ERR_INVALID_ARG;
+    if (!cplan || !C || !aligned16(C)) return FMM_ERR_INVALID_ARG;
     fmm_plan* plan = const_cast<fmm_plan*>(cplan);
     FmmLayout L;
     fmm_status_t s = check_ws(plan, M, N, K, ws, ws_bytes, &L);
@@ -417,7 +420,7 @@ fmm_status_t fmm_multiply_only(const fmm_plan_t* cplan, float* C, int64_t M, int
 fmm_status_t fmm_matmul(const fmm_plan_t* cplan, const float* A, const float* B, float* C,
                         int64_t M, int64_t N, int64_t K, void* ws, size_t ws_bytes, void* stream)
 {
-    if (!cplan || !A || !B || !C) return FMM_ERR_INVALID_ARG;
+    if (!cplan || !A || !B || !C || !aligned16(A) || !aligned16(B) || !aligned16(C)) return FMM_ERR_INVALID_ARG;
     fmm_plan* plan = const_cast<fmm_plan*>(cplan);
     FmmLayout L;
     fmm_status_t s = check_ws(plan, M, N, K, ws, ws_bytes, &L);

@@ -30,6 +30,17 @@ def test_matmul_rejects_bad_shapes_workspace_and_pointers():
     assert call(256, 256, 256, None, ws.numel()) == 4
     assert call(256, 256, 256, C.c_void_p(ws.data_ptr() + 8), ws.numel()) == 4   # misaligned
     assert call(256, 256, 256, p(ws), ws.numel(), A=None) == 1
+    # operands that are not 16-byte aligned are refused before anything is launched (the kernels use vector loads)
+    big = torch.zeros(256 * 256 + 4, device="cuda")
+    odd = lambda off: C.c_void_p(big.data_ptr() + off)
+    assert lib.fmm_matmul(plan._h, odd(4), p(a), p(c), C.c_int64(256), C.c_int64(256), C.c_int64(256), p(ws),
+                          C.c_size_t(ws.numel()), None) == 1
+    assert lib.fmm_matmul(plan._h, p(a), odd(8), p(c), C.c_int64(256), C.c_int64(256), C.c_int64(256), p(ws),
+                          C.c_size_t(ws.numel()), None) == 1
+    assert lib.fmm_matmul(plan._h, p(a), p(a), odd(4), C.c_int64(256), C.c_int64(256), C.c_int64(256), p(ws),
+                          C.c_size_t(ws.numel()), None) == 1
+    assert lib.fmm_matmul(plan._h, odd(16), p(a), p(c), C.c_int64(256), C.c_int64(256), C.c_int64(256), p(ws),
+                          C.c_size_t(ws.numel()), None) == 0
     need = C.c_size_t()
     assert lib.fmm_workspace_bytes(plan._h, C.c_int64(100), C.c_int64(256), C.c_int64(256), C.byref(need)) == 2
     torch.cuda.synchronize()
