@@ -440,17 +440,37 @@ __global__ void __launch_bounds__(256) encode2_b_kernel(const EncodeParams p)
     const int kb = blockIdx.y;                                      // 32-k block
     const int k0 = kb * 32 + (lane & 7) * 4;
     const int b = blockIdx.z;
-    const float* base = p.in + (int64_t)b * p.in_batch_stride + (int64_t)k0 * p.ld + j;
     const int64_t term_codes = (int64_t)p.rows * p.cols;
     const int my_r = lane & 7;
+    // The block's 32 k x 32 columns of each of the 16 sub-blocks go through shared memory: the global loads are
+    // whole 128-byte row segments (a thread reading its own 4 k x 1 column directly touches eight lines per warp
+    // instruction with 16 bytes each and is bound by L1 wavefronts), the transposed reads are conflict-free with
+    // rows padded to 33 words.  Two passes of eight sub-blocks keep the buffer under the static 48 KB.
+    __shared__ float tile[8][32][33];
     float4 raw[4][4];
+    {
+        const int lrow = threadIdx.x >> 3, lc = (threadIdx.x & 7) * 4;
+        const float* blk = p.in + (int64_t)b * p.in_batch_stride + ((int64_t)kb * 32 + lrow) * p.ld + blockIdx.x * 32 + lc;
+        const int rk = (lane & 7) * 4, rc = warp * 4 + (lane >> 3);
 #pragma unroll
-    for (int q1 = 0; q1 < 4; ++q1)
+        for (int pass = 0; pass < 2; ++pass) {
+            if (pass) __syncthreads();
+            float4 v[8];
 #pragma unroll
-        for (int q2 = 0; q2 < 4; ++q2) {
-            const float* src = base + p.qoff_outer[q1] + p.qoff[q2];
-            raw[q1][q2] = make_float4(__ldg(src), __ldg(src + p.ld), __ldg(src + 2 * p.ld), __ldg(src + 3 * p.ld));
+            for (int sblk = 0; sblk < 8; ++sblk)
+                v[sblk] = __ldg(reinterpret_cast<const float4*>(blk + p.qoff_outer[2 * pass + (sblk >> 2)] + p.qoff[sblk & 3]));
+#pragma unroll
+            for (int sblk = 0; sblk < 8; ++sblk) {
+                tile[sblk][lrow][lc] = v[sblk].x; tile[sblk][lrow][lc + 1] = v[sblk].y;
+                tile[sblk][lrow][lc + 2] = v[sblk].z; tile[sblk][lrow][lc + 3] = v[sblk].w;
+            }
+            __syncthreads();
+#pragma unroll
+            for (int sblk = 0; sblk < 8; ++sblk)
+                raw[2 * pass + (sblk >> 2)][sblk & 3] = make_float4(tile[sblk][rk][rc], tile[sblk][rk + 1][rc],
+                                                                    tile[sblk][rk + 2][rc], tile[sblk][rk + 3][rc]);
         }
+    }
 #pragma unroll
     for (int r1 = 0; r1 < FMM_MAX_RANK; ++r1) {
         if (row_used<NZ>(r1, p.R)) {
