@@ -46,3 +46,72 @@ def test_full_size_operands_bit_exact_and_sampled_rows_of_c(mode, blk):
         rel = np.linalg.norm(block - want) / np.linalg.norm(want)
         assert rel <= 1e-5, f"quadrant {q}: sampled rows differ by {rel:.3e}"
     assert np.isfinite(got).all()
+
+
+def test_full_size_two_levels_operands_bit_exact_and_sampled_rows_of_c():
+    # n = 8192 at two recursion levels (49 leaf products of 2048^3; fused two-level encoders, term groups as work
+    # items, outer decoder as a separate kernel): all leaf operands in full, C on sampled leaf rows of all 16 blocks
+    n, blk, mode = 8192, 32, "ue8m0"
+    leaf = n // 4
+    A, B = Wl.gaussian(n, n, n, seed=0)
+    plan = make_plan("phi_optimal", 2, blk, mode)
+    ws = plan.workspace(n, n, n)
+    C = plan.matmul(dev(A), dev(B), workspace=ws)
+    torch.cuda.synchronize()
+    assert plan.device_status() == (0, 0)
+    U, V, W = coeffs("phi_optimal")
+    ca, sa, ea = O.encode(A, "A", U, V, 2, blk, MODES[mode])
+    cb, sb, eb = O.encode(B, "B", U, V, 2, blk, MODES[mode])
+    assert len(ca) == 49
+    rng = np.random.default_rng(2)
+    rows = np.sort(rng.choice(leaf, size=12, replace=False))
+    Mrows = []
+    for t in range(49):                                  # t = 7 * (outer term) + (inner term)
+        qa, sca = plan.quantized_operand(ws, n, n, n, t, "A")
+        qb, scb = plan.quantized_operand(ws, n, n, n, t, "B")
+        assert np.array_equal(qa, ca[t]) and np.array_equal(qb, cb[t]), f"codes differ in term {t}"
+        assert np.array_equal(sca, ea[t]) and np.array_equal(scb, eb[t]), f"scales differ in term {t}"
+        Mrows.append(O.dequant_rows(ca[t][rows], sa[t][rows], blk) @ O.dequant_cols(cb[t], sb[t], blk))
+    got = C.cpu().numpy().astype(np.float64)
+    assert np.isfinite(got).all()
+    for q1 in range(4):
+        for q2 in range(4):
+            want = sum(float(W[t1][q1]) * float(W[t2][q2]) * Mrows[7 * t1 + t2] for t1 in range(7) for t2 in range(7)
+                       if W[t1][q1] != 0 and W[t2][q2] != 0)
+            r0 = (q1 >> 1) * 2 * leaf + (q2 >> 1) * leaf
+            c0 = (q1 & 1) * 2 * leaf + (q2 & 1) * leaf
+            block = got[r0 + rows][:, c0:c0 + leaf]
+            rel = np.linalg.norm(block - want) / np.linalg.norm(want)
+            assert rel <= 1e-5, f"block ({q1},{q2}): sampled rows differ by {rel:.3e}"
+
+
+def test_full_size_rectangular_llm_shape_sampled_rows_of_c():
+    # M, K, N = 16384, 8192, 8192 with per-column outlier channels in A and small-variance weights in B: the quantized
+    # operands in full, C on sampled rows of each output block
+    M, K, N, blk, mode = 16384, 8192, 8192, 32, "fp32"
+    A, B = Wl.FAMILIES["llm"](M, K, N, seed=3)
+    plan = make_plan("strassen", 1, blk, mode)
+    ws = plan.workspace(M, N, K)
+    C = plan.matmul(dev(A), dev(B), workspace=ws)
+    torch.cuda.synchronize()
+    assert plan.device_status() == (0, 0)
+    U, V, W = coeffs("strassen")
+    ca, sa, _ = O.encode(A, "A", U, V, 1, blk, MODES[mode])
+    cb, sb, _ = O.encode(B, "B", U, V, 1, blk, MODES[mode])
+    rng = np.random.default_rng(4)
+    rows = np.sort(rng.choice(M // 2, size=16, replace=False))
+    Mrows = []
+    for t in range(7):
+        qa, sca = plan.quantized_operand(ws, M, N, K, t, "A")
+        qb, scb = plan.quantized_operand(ws, M, N, K, t, "B")
+        assert np.array_equal(qa, ca[t]) and np.array_equal(qb, cb[t]), f"codes differ in term {t}"
+        assert np.array_equal(sca, sa[t]) and np.array_equal(scb, sb[t]), f"scales differ in term {t}"
+        Mrows.append(O.dequant_rows(ca[t][rows], sa[t][rows], blk) @ O.dequant_cols(cb[t], sb[t], blk))
+    got = C.cpu().numpy().astype(np.float64)
+    assert np.isfinite(got).all()
+    for q in range(4):
+        want = sum(float(W[r][q]) * Mrows[r] for r in range(7) if W[r][q] != 0)
+        r0, c0 = (q >> 1) * (M // 2), (q & 1) * (N // 2)
+        block = got[r0 + rows][:, c0:c0 + N // 2]
+        rel = np.linalg.norm(block - want) / np.linalg.norm(want)
+        assert rel <= 1e-5, f"quadrant {q}: sampled rows differ by {rel:.3e}"
