@@ -53,6 +53,24 @@ def test_algorithmic_work_matches_the_derivation():
     assert (enc0 + gemm0) / 1e6 == pytest.approx(1107, rel=5e-3)
 
 
+def test_combined_roofline_time_follows_the_derivation():
+    # n = 8192, one level: tensor phase at the given fp8 peak, or the fp32 promotion bound (2 lane-ops per element
+    # and 32-k block on 148 x 128 lanes at 1.965 GHz) if larger, plus the algorithmic bytes at the given bandwidth
+    n, peak, bw = 8192, 3293.6, 6459.0
+    flops, enc, gemm = bench.algorithmic_work(n, n, n, 1, 7, 1, 32)
+    want = (flops / (peak * 1e12) + (enc + gemm) / (bw * 1e9)) * 1e3
+    assert bench.combined_roofline_ms(n, n, n, 1, 7, "ue8m0", 32, peak, bw) == pytest.approx(want, rel=1e-12)
+    flops, enc, gemm = bench.algorithmic_work(n, n, n, 1, 7, 4, 32)
+    alu = 2.0 * n * n * (n / 32) * (7 / 8) / (148 * 128 * 1.965e9)
+    assert alu > flops / (peak * 1e12)
+    want = (alu + (enc + gemm) / (bw * 1e9)) * 1e3
+    assert bench.combined_roofline_ms(n, n, n, 1, 7, "fp32", 32, peak, bw) == pytest.approx(want, rel=1e-12)
+    # weight tiles: one FMA per element and 128-k block, so the tensor phase is the larger term again
+    t = bench.combined_roofline_ms(n, n, n, 1, 7, "fp32+tile128", 128, peak, bw)
+    flops, enc, gemm = bench.algorithmic_work(n, n, n, 1, 7, 4, 128)
+    assert t == pytest.approx((flops / (peak * 1e12) + (enc + gemm) / (bw * 1e9)) * 1e3, rel=1e-12)
+
+
 def test_reference_arm_prints_one_json_line():
     out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--steps", "1",
                           "--warmup", "0", "--ref-n", "256"], capture_output=True, text=True, timeout=300)
