@@ -45,7 +45,8 @@ typedef enum {
     FMM_ERR_ALLOC = 5,          /* host or device allocation failed (plan creation only) */
     FMM_ERR_CUDA = 6,           /* a CUDA runtime / driver call failed (no device, bad stream, ...) */
     FMM_ERR_ARCH = 7,           /* current device is not compute capability 10.x */
-    FMM_ERR_DEVICE_TIMEOUT = 8  /* a bounded device-side wait gave up (see fmm_device_status) */
+    FMM_ERR_DEVICE_TIMEOUT = 8, /* a bounded device-side wait gave up (see fmm_device_status) */
+    FMM_ERR_WRONG_DEVICE = 9    /* the current CUDA device is not the one the plan was created on */
 } fmm_status_t;
 
 typedef enum {
@@ -103,7 +104,10 @@ fmm_status_t fmm_workspace_bytes(const fmm_plan_t* plan, int64_t M, int64_t N, i
  *   (hence of block_k); otherwise FMM_ERR_SHAPE.
  *   workspace dev, 1024-byte aligned, at least fmm_workspace_bytes() bytes, caller-owned; its
  *   contents after the call are the quantized operands (see fmm_quantized_view).
- * Asynchronous on cuda_stream.  Calls sharing a plan or a workspace must be stream-ordered. */
+ *   The plan's device (the one current at fmm_plan_create) must be the current device: FMM_ERR_WRONG_DEVICE otherwise;
+ *   the same holds for every call that takes a plan and touches the device.
+ * Asynchronous on cuda_stream.  Calls sharing a workspace must be stream-ordered; a plan may be shared by host
+ * threads (it is read-only during a call, apart from the launch counter below). */
 fmm_status_t fmm_matmul(const fmm_plan_t* plan, const float* A, const float* B, float* C,
                         int64_t M, int64_t N, int64_t K, void* workspace, size_t workspace_bytes,
                         void* cuda_stream);
@@ -116,7 +120,8 @@ fmm_status_t fmm_matmul(const fmm_plan_t* plan, const float* A, const float* B, 
  * Everything is enqueued on cuda_stream in order (upload A, upload B, product, download C) and nothing is
  * synchronised: C is valid once the stream has drained.  Calls on different streams with different workspaces
  * overlap one call's uploads with another's product and download (the links are full duplex); that is the
- * intended use for a sequence of products.  Errors as fmm_matmul. */
+ * intended use for a sequence of products.  Errors as fmm_matmul, except that the host pointers need no
+ * particular alignment; fmm_host_workspace_bytes returns FMM_ERR_INVALID_ARG for a null plan or bytes. */
 fmm_status_t fmm_host_workspace_bytes(const fmm_plan_t* plan, int64_t M, int64_t N, int64_t K,
                                       size_t* bytes);
 fmm_status_t fmm_matmul_host(const fmm_plan_t* plan, const float* A, const float* B, float* C,
@@ -178,12 +183,13 @@ fmm_status_t fmm_error_stats_noalloc(const float* C, const double* Cref, int64_t
                                      double* out3, void* cuda_stream);
 int64_t fmm_error_stats_noalloc_max_elements(void);
 
-/* Reads the plan's device status word (synchronises the device).  *code == 0: no bounded wait has
+/* Reads the plan's device status word after cudaDeviceSynchronize (all streams of the device, non-blocking
+ * ones included, have drained).  *code == 0: no bounded wait has
  * given up since plan creation; otherwise a kernel-specific location code, and the results of the
  * call that set it are invalid.  Returns FMM_ERR_DEVICE_TIMEOUT when *code != 0. */
 fmm_status_t fmm_device_status(const fmm_plan_t* plan, int* code);
 
-/* Resets the plan's status words to zero (synchronises the device). */
+/* Resets the plan's status words to zero, after cudaDeviceSynchronize. */
 fmm_status_t fmm_device_status_clear(const fmm_plan_t* plan);
 
 /* Self-test of the failure-detection path (no counterpart in the paper): enqueues a one-warp kernel that
@@ -202,7 +208,8 @@ fmm_status_t fmm_phi_gamma(int rank, const float* U, const float* V, const float
 fmm_status_t fmm_brent_residual(int rank, const float* U, const float* V, const float* W,
                                 double* max_residual);
 
-/* Number of kernels the last fmm_matmul / fmm_encode_only / fmm_multiply_only on this plan launched. */
+/* Number of kernels the last fmm_matmul / fmm_encode_only / fmm_multiply_only on this plan launched (with several
+ * host threads on one plan: of whichever call finished last). */
 fmm_status_t fmm_last_launch_count(const fmm_plan_t* plan, int* launches);
 
 const char* fmm_status_string(fmm_status_t status);

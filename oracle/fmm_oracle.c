@@ -456,6 +456,33 @@ int oracle_fused_fmm_ex(const float *A, const float *B, double *C,
     return 0;
 }
 
+/* Selected entries of one leaf product from already quantized operands (for sampled checks at sizes
+ * where the whole product is too slow).  ca [m x k] codes and sa [m x k/blk] scales of the A-side
+ * combination, cb [k x n] codes and sb [k/blk x n] scales of the B-side one, as oracle_encode returns
+ * them.  out[s * ncols + t] = sum_p deq_a(rows[s], p) * deq_b(p, cols[t]) with the same exact fp64
+ * dequantization and the same summation order over p as leaf_product / gemm_f64. */
+void oracle_leaf_product_sample(const uint8_t *ca, const float *sa, const uint8_t *cb, const float *sb,
+                                int64_t m, int64_t n, int64_t k, int blk,
+                                const int64_t *rows, int64_t nrows, const int64_t *cols, int64_t ncols,
+                                double *out)
+{
+    (void)m;
+    int64_t nb = k / blk;
+#pragma omp parallel for schedule(static)
+    for (int64_t s = 0; s < nrows; ++s) {
+        int64_t i = rows[s];
+        double *c = out + s * ncols;
+        for (int64_t t = 0; t < ncols; ++t) c[t] = 0.0;
+        for (int64_t p = 0; p < k; ++p) {
+            double a = oracle_e4m3_decode(ca[i * k + p]) * (double)sa[i * nb + p / blk];
+            for (int64_t t = 0; t < ncols; ++t) {
+                int64_t j = cols[t];
+                c[t] += a * (oracle_e4m3_decode(cb[p * n + j]) * (double)sb[(p / blk) * n + j]);
+            }
+        }
+    }
+}
+
 /* ------------------------------- quantized leaf operands, for bit parity */
 
 static void encode_rec(const realization_t *D, int levels, int side,

@@ -186,6 +186,24 @@ def ref_gemm_rows(A, B, rows):
     return out
 
 
+def leaf_product_sample(codes_a, scales_a, codes_b, scales_b, blk, rows, cols):
+    """Entries (rows x cols) of one leaf product S^ T^ in fp64 from the quantized operands of one term as
+    `encode` returns them (A side [m, k] / [m, k/blk], B side [k, n] / [k/blk, n]); plain loops in C."""
+    ca = np.ascontiguousarray(codes_a, dtype=np.uint8)
+    cb = np.ascontiguousarray(codes_b, dtype=np.uint8)
+    sa, sb = _f32(scales_a), _f32(scales_b)
+    m, k = ca.shape
+    k2, n = cb.shape
+    assert k == k2 and sa.shape == (m, k // blk) and sb.shape == (k // blk, n)
+    rows = np.ascontiguousarray(np.asarray(rows, dtype=np.int64))
+    cols = np.ascontiguousarray(np.asarray(cols, dtype=np.int64))
+    out = np.empty((rows.size, cols.size), np.float64)
+    lib().oracle_leaf_product_sample(_p(ca), _p(sa), _p(cb), _p(sb), C.c_int64(m), C.c_int64(n), C.c_int64(k),
+                                     C.c_int(blk), _p(rows), C.c_int64(rows.size), _p(cols), C.c_int64(cols.size),
+                                     _p(out))
+    return out
+
+
 def error_stats(Cm, Cref):
     """[sum (C-Cref)^2, sum Cref^2, max |C-Cref|] in fp64."""
     Cm = np.ascontiguousarray(np.asarray(Cm, dtype=np.float64))

@@ -222,3 +222,79 @@ def act(U, V, W, X, Y, Z):
     w = from_cyclic(W)          # the swap of entries 12 and 21 is its own inverse
     return (_rowmat(U, _kron2(X, _inv_t(Y))), _rowmat(V, _kron2(Y, _inv_t(Z))),
             from_cyclic(_rowmat(w, _kron2(Z, _inv_t(X)))))
+
+
+class _Jet:
+    """c0 + c1 s + c2 s^2 (higher powers of s dropped), coefficients in Q(sqrt 3)."""
+    __slots__ = ("c",)
+
+    def __init__(self, c0=0, c1=0, c2=0):
+        self.c = (Q3.of(c0), Q3.of(c1), Q3.of(c2))
+
+    @staticmethod
+    def of(x):
+        return x if isinstance(x, _Jet) else _Jet(x)
+
+    def __add__(self, o):
+        o = _Jet.of(o)
+        return _Jet(*(a + b for a, b in zip(self.c, o.c)))
+
+    __radd__ = __add__
+
+    def __mul__(self, o):
+        o = _Jet.of(o)
+        a, b = self.c, o.c
+        return _Jet(a[0] * b[0], a[0] * b[1] + a[1] * b[0], a[0] * b[2] + a[1] * b[1] + a[2] * b[0])
+
+    __rmul__ = __mul__
+
+
+def phi_second_order(U, V, W, direction):
+    """Exact coefficient of s^2 in Phi(D . (e^{s H_X}, e^{s H_Y}, e^{s H_Z})) (App. A, second-order form),
+    with direction = (x1, y1, z1, x2, y2, z2) rational and H(p, q) = 1/2 [[p, q], [q, -p]].
+    H is symmetric, so e^{sH} = I + sH + s^2 H^2 / 2 + ... and (e^{sH})^-T = e^{-sH}; terms beyond s^2
+    cannot reach the coefficient, which makes a truncated series exact."""
+    x1, y1, z1, x2, y2, z2 = (Fr(d) for d in direction)
+
+    def expo(p, q, sign):
+        h = [[p / 2, q / 2], [q / 2, -p / 2]]
+        h2 = [[sum(h[i][k] * h[k][j] for k in range(2)) for j in range(2)] for i in range(2)]
+        return [[_Jet(1 if i == j else 0, sign * h[i][j], h2[i][j] / 2) for j in range(2)] for i in range(2)]
+
+    X, Xi = expo(x1, x2, 1), expo(x1, x2, -1)
+    Y, Yi = expo(y1, y2, 1), expo(y1, y2, -1)
+    Z, Zi = expo(z1, z2, 1), expo(z1, z2, -1)
+
+    def kron(A, B):
+        return [[A[i][j] * B[k][l] for j in range(2) for l in range(2)] for i in range(2) for k in range(2)]
+
+    def rows_times(rows, M):
+        out = []
+        for r in rows:
+            out.append([sum((_Jet.of(r[j]) * M[j][q] for j in range(4)), _Jet()) for q in range(4)])
+        return out
+
+    def sq(row):
+        return sum((x * x for x in row), _Jet())
+
+    U2 = rows_times(U, kron(X, Yi))
+    V2 = rows_times(V, kron(Y, Zi))
+    w2 = rows_times(from_cyclic(W), kron(Z, Xi))        # squared row norms do not depend on the entry order
+    total = _Jet()
+    for r in range(len(U)):
+        total = total + sq(U2[r]) * sq(V2[r]) * sq(w2[r])
+    return total.c
+
+
+def phi_hessian(U, V, W):
+    """6 x 6 matrix of second derivatives of Phi at the realization in the coordinates t of App. A
+    (exact, by polarization of phi_second_order): Phi_t = Phi + g.t + 1/2 t^T Hess t + O(|t|^3)."""
+    e = [[1 if i == j else 0 for j in range(6)] for i in range(6)]
+    diag = [phi_second_order(U, V, W, e[i])[2] for i in range(6)]
+    Hs = [[None] * 6 for _ in range(6)]
+    for i in range(6):
+        Hs[i][i] = diag[i] * 2
+        for j in range(i + 1, 6):
+            both = phi_second_order(U, V, W, [e[i][k] + e[j][k] for k in range(6)])[2]
+            Hs[i][j] = Hs[j][i] = both - diag[i] - diag[j]
+    return Hs

@@ -79,10 +79,20 @@ void make_layout(const fmm_plan* plan, int64_t M, int64_t N, int64_t K, FmmLayou
 // the kernels read the operands with 16-byte vector loads and write C through a tensor map
 bool aligned16(const void* p) { return ((uintptr_t)p & 15) == 0; }
 
+// a plan's device tables live on the device that was current at fmm_plan_create
+fmm_status_t check_device(const fmm_plan* plan)
+{
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return FMM_ERR_CUDA; }
+    return dev == plan->device ? FMM_OK : FMM_ERR_WRONG_DEVICE;
+}
+
 fmm_status_t check_ws(const fmm_plan* plan, int64_t M, int64_t N, int64_t K, void* ws, size_t ws_bytes,
                       FmmLayout* L)
 {
-    fmm_status_t s = check_shape(plan, M, N, K);
+    fmm_status_t s = check_device(plan);
+    if (s != FMM_OK) return s;
+    s = check_shape(plan, M, N, K);
     if (s != FMM_OK) return s;
     make_layout(plan, M, N, K, L);
     if (!ws || ((uintptr_t)ws & 1023) || ws_bytes < L->total) return FMM_ERR_WORKSPACE;
@@ -97,8 +107,8 @@ void fill_coef(float dst[FMM_MAX_RANK][4], const float src[FMM_MAX_RANK][4], int
 }
 
 // One side of steps 1-2: outer levels as fp32 combinations, last level fused with the quantizer.
-fmm_status_t encode_side(fmm_plan* plan, const FmmLayout& L, char* ws, const float* X,
-                         int64_t rows, int64_t cols, bool b_side, cudaStream_t st)
+fmm_status_t encode_side(const fmm_plan* plan, const FmmLayout& L, char* ws, const float* X,
+                         int64_t rows, int64_t cols, bool b_side, cudaStream_t st, int* launches)
 {
     const int R = plan->rank, lv = plan->levels;
     const int blk = plan->qp.block_k, mode = (int)plan->qp.scale_mode;
@@ -156,7 +166,7 @@ fmm_status_t encode_side(fmm_plan* plan, const FmmLayout& L, char* ws, const flo
             c.out = reinterpret_cast<float*>(ws + (b_side ? L.inter_b[level] : L.inter_a[level]));
             s = fmm_launch_comb(c, st);
             if (s != FMM_OK) return s;
-            plan->last_launches++;
+            ++*launches;
             cur = c.out; cur_rows /= 2; cur_cols /= 2; cur_ld = cur_cols; cur_stride = cur_rows * cur_cols;
             batch *= R;
         }
@@ -169,17 +179,17 @@ fmm_status_t encode_side(fmm_plan* plan, const FmmLayout& L, char* ws, const flo
         e.s_step = 0; e.s_ld = e.cols; e.sf_blocks = (b_side ? e.cols : e.rows) / 128;
         if (fused2) {
             s = b_side ? fmm_launch_encode2_b(e, mode, st) : fmm_launch_encode2_a(e, blk, mode, st);
-            if (s == FMM_OK) plan->last_launches++;
+            if (s == FMM_OK) ++*launches;
             return s;
         }
     }
     s = b_side ? fmm_launch_encode_b(e, blk, mode, st) : fmm_launch_encode_a(e, blk, mode, st);
-    if (s == FMM_OK) plan->last_launches++;
+    if (s == FMM_OK) ++*launches;
     return s;
 }
 
-fmm_status_t multiply(fmm_plan* plan, const FmmLayout& L, char* ws, float* C, int64_t M, int64_t N,
-                      cudaStream_t st)
+fmm_status_t multiply(const fmm_plan* plan, const FmmLayout& L, char* ws, float* C, int64_t M, int64_t N,
+                      cudaStream_t st, int* launches)
 {
     GemmParams g;
     memset(&g, 0, sizeof(g));
@@ -201,9 +211,7 @@ fmm_status_t multiply(fmm_plan* plan, const FmmLayout& L, char* ws, float* C, in
     g.terms_per_group = plan->levels >= 2 ? plan->rank : (int)L.terms;
     g.out_start = plan->d_out_start; g.out = plan->d_out; g.status = plan->d_status;
     g.sb_tile = plan->qp.b_tile_n == 128 ? 1 : 0;
-    int launches = 0;
-    fmm_status_t s = fmm_launch_gemm(g, plan->qp.block_k, (int)plan->qp.scale_mode, st, &launches);
-    plan->last_launches += launches;
+    fmm_status_t s = fmm_launch_gemm(g, plan->qp.block_k, (int)plan->qp.scale_mode, st, launches);
     if (s != FMM_OK) return s;
     for (int l = lv - 1; l >= 1; --l) {
         DecodeParams d;
@@ -216,7 +224,7 @@ fmm_status_t multiply(fmm_plan* plan, const FmmLayout& L, char* ws, float* C, in
             for (int q = 0; q < 4; ++q) d.W[r][q] = plan->W[r][q];
         s = fmm_launch_decode(d, st);
         if (s != FMM_OK) return s;
-        plan->last_launches++;
+        ++*launches;
     }
     return FMM_OK;
 }
@@ -237,6 +245,7 @@ const char* fmm_status_string(fmm_status_t s)
         case FMM_ERR_CUDA: return "CUDA call failed";
         case FMM_ERR_ARCH: return "device is not compute capability 10.x (B200)";
         case FMM_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait timed out";
+        case FMM_ERR_WRONG_DEVICE: return "the current device is not the one the plan was created on";
     }
     return "unknown status";
 }
@@ -294,7 +303,8 @@ fmm_status_t fmm_plan_create(fmm_plan_t** out, int rank, const float* U, const f
 
     fmm_plan* p = new (std::nothrow) fmm_plan;
     if (!p) return FMM_ERR_ALLOC;
-    memset(p, 0, sizeof(*p));
+    memset(static_cast<void*>(p), 0, sizeof(*p));
+    p->last_launches.store(0, std::memory_order_relaxed);
     p->rank = rank; p->levels = levels; p->qp = *qp; p->device = dev;
     if (levels > 0)
         for (int r = 0; r < rank; ++r)
@@ -390,48 +400,48 @@ fmm_status_t fmm_quantized_view(const fmm_plan_t* plan, int64_t M, int64_t N, in
     return FMM_OK;
 }
 
-fmm_status_t fmm_encode_only(const fmm_plan_t* cplan, const float* A, const float* B, int64_t M, int64_t N, int64_t K,
+fmm_status_t fmm_encode_only(const fmm_plan_t* plan, const float* A, const float* B, int64_t M, int64_t N, int64_t K,
                              void* ws, size_t ws_bytes, void* stream)
 {
-    if (!cplan || !A || !B || !aligned16(A) || !aligned16(B)) return FMM_ERR_INVALID_ARG;
-    fmm_plan* plan = const_cast<fmm_plan*>(cplan);
+    if (!plan || !A || !B || !aligned16(A) || !aligned16(B)) return FMM_ERR_INVALID_ARG;
     FmmLayout L;
     fmm_status_t s = check_ws(plan, M, N, K, ws, ws_bytes, &L);
     if (s != FMM_OK) return s;
-    plan->last_launches = 0;
+    int launches = 0;
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
-    s = encode_side(plan, L, static_cast<char*>(ws), A, M, K, false, st);
-    if (s != FMM_OK) return s;
-    return encode_side(plan, L, static_cast<char*>(ws), B, K, N, true, st);
+    s = encode_side(plan, L, static_cast<char*>(ws), A, M, K, false, st, &launches);
+    if (s == FMM_OK) s = encode_side(plan, L, static_cast<char*>(ws), B, K, N, true, st, &launches);
+    plan->last_launches.store(launches, std::memory_order_relaxed);
+    return s;
 }
 
-fmm_status_t fmm_multiply_only(const fmm_plan_t* cplan, float* C, int64_t M, int64_t N, int64_t K,
+fmm_status_t fmm_multiply_only(const fmm_plan_t* plan, float* C, int64_t M, int64_t N, int64_t K,
                                void* ws, size_t ws_bytes, void* stream)
 {
-    if (!cplan || !C || !aligned16(C)) return FMM_ERR_INVALID_ARG;
-    fmm_plan* plan = const_cast<fmm_plan*>(cplan);
+    if (!plan || !C || !aligned16(C)) return FMM_ERR_INVALID_ARG;
     FmmLayout L;
     fmm_status_t s = check_ws(plan, M, N, K, ws, ws_bytes, &L);
     if (s != FMM_OK) return s;
-    plan->last_launches = 0;
-    return multiply(plan, L, static_cast<char*>(ws), C, M, N, reinterpret_cast<cudaStream_t>(stream));
+    int launches = 0;
+    s = multiply(plan, L, static_cast<char*>(ws), C, M, N, reinterpret_cast<cudaStream_t>(stream), &launches);
+    plan->last_launches.store(launches, std::memory_order_relaxed);
+    return s;
 }
 
-fmm_status_t fmm_matmul(const fmm_plan_t* cplan, const float* A, const float* B, float* C,
+fmm_status_t fmm_matmul(const fmm_plan_t* plan, const float* A, const float* B, float* C,
                         int64_t M, int64_t N, int64_t K, void* ws, size_t ws_bytes, void* stream)
 {
-    if (!cplan || !A || !B || !C || !aligned16(A) || !aligned16(B) || !aligned16(C)) return FMM_ERR_INVALID_ARG;
-    fmm_plan* plan = const_cast<fmm_plan*>(cplan);
+    if (!plan || !A || !B || !C || !aligned16(A) || !aligned16(B) || !aligned16(C)) return FMM_ERR_INVALID_ARG;
     FmmLayout L;
     fmm_status_t s = check_ws(plan, M, N, K, ws, ws_bytes, &L);
     if (s != FMM_OK) return s;
-    plan->last_launches = 0;
+    int launches = 0;
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
-    s = encode_side(plan, L, static_cast<char*>(ws), A, M, K, false, st);
-    if (s != FMM_OK) return s;
-    s = encode_side(plan, L, static_cast<char*>(ws), B, K, N, true, st);
-    if (s != FMM_OK) return s;
-    return multiply(plan, L, static_cast<char*>(ws), C, M, N, st);
+    s = encode_side(plan, L, static_cast<char*>(ws), A, M, K, false, st, &launches);
+    if (s == FMM_OK) s = encode_side(plan, L, static_cast<char*>(ws), B, K, N, true, st, &launches);
+    if (s == FMM_OK) s = multiply(plan, L, static_cast<char*>(ws), C, M, N, st, &launches);
+    plan->last_launches.store(launches, std::memory_order_relaxed);
+    return s;
 }
 
 // Host-operand variant: [product workspace | A | B | C] in the caller's device buffer, 1024-byte aligned parts.
@@ -439,6 +449,7 @@ static size_t host_align(size_t x) { return (x + 1023) & ~(size_t)1023; }
 
 fmm_status_t fmm_host_workspace_bytes(const fmm_plan_t* plan, int64_t M, int64_t N, int64_t K, size_t* bytes)
 {
+    if (!bytes) return FMM_ERR_INVALID_ARG;
     size_t ws = 0;
     fmm_status_t s = fmm_workspace_bytes(plan, M, N, K, &ws);
     if (s != FMM_OK) return s;
@@ -477,23 +488,22 @@ fmm_status_t fmm_matmul_host(const fmm_plan_t* plan, const float* A, const float
 fmm_status_t fmm_device_status(const fmm_plan_t* plan, int* code)
 {
     if (!plan || !code) return FMM_ERR_INVALID_ARG;
+    fmm_status_t sd = check_device(plan);
+    if (sd != FMM_OK) return sd;
     int h[4] = {0, 0, 0, 0};
+    // every stream, including non-blocking ones that the copy below would not wait for
+    if (cudaDeviceSynchronize() != cudaSuccess) { cudaGetLastError(); return FMM_ERR_CUDA; }
     if (cudaMemcpy(h, plan->d_status, sizeof(h), cudaMemcpyDeviceToHost) != cudaSuccess) { cudaGetLastError(); return FMM_ERR_CUDA; }
     *code = h[0];
     return h[0] ? FMM_ERR_DEVICE_TIMEOUT : FMM_OK;
 }
 
-#ifdef FMM_TIMING
-// experiment builds only: raw copy of the status / timing words
-fmm_status_t fmm_debug_status64(const fmm_plan_t* plan, int* out64)
-{
-    return cudaMemcpy(out64, plan->d_status, 64 * sizeof(int), cudaMemcpyDeviceToHost) == cudaSuccess ? FMM_OK : FMM_ERR_CUDA;
-}
-#endif
-
 fmm_status_t fmm_device_status_clear(const fmm_plan_t* plan)
 {
     if (!plan) return FMM_ERR_INVALID_ARG;
+    fmm_status_t sd = check_device(plan);
+    if (sd != FMM_OK) return sd;
+    if (cudaDeviceSynchronize() != cudaSuccess) { cudaGetLastError(); return FMM_ERR_CUDA; }
     if (cudaMemset(plan->d_status, 0, 64 * sizeof(int)) != cudaSuccess) { cudaGetLastError(); return FMM_ERR_CUDA; }
     return FMM_OK;
 }
@@ -501,13 +511,15 @@ fmm_status_t fmm_device_status_clear(const fmm_plan_t* plan)
 fmm_status_t fmm_selftest_bounded_wait(const fmm_plan_t* plan, int64_t limit_ns, void* stream)
 {
     if (!plan || limit_ns <= 0 || limit_ns > 2000000000ll) return FMM_ERR_INVALID_ARG;
+    fmm_status_t sd = check_device(plan);
+    if (sd != FMM_OK) return sd;
     return fmm_launch_bounded_wait_selftest(plan->d_status, (unsigned long long)limit_ns, reinterpret_cast<cudaStream_t>(stream));
 }
 
 fmm_status_t fmm_last_launch_count(const fmm_plan_t* plan, int* launches)
 {
     if (!plan || !launches) return FMM_ERR_INVALID_ARG;
-    *launches = plan->last_launches;
+    *launches = plan->last_launches.load(std::memory_order_relaxed);
     return FMM_OK;
 }
 

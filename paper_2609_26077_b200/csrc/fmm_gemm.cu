@@ -108,14 +108,6 @@ struct Cfg {
     static_assert(!MX || BN + STAGES * SF_COLS <= 512, "TMEM budget");
 };
 
-#ifdef FMM_TIMING
-#define TCLK() clock64()
-#define TADD(slot, t0) do { if (blockIdx.x == 0 && lane == 0) tim[slot] += clock64() - (t0); } while (0)
-#else
-#define TCLK() 0ll
-#define TADD(slot, t0) do { (void)(t0); } while (0)
-#endif
-
 constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;   // 2 s: far beyond any legitimate wait
 
 struct Ctl {
@@ -206,10 +198,6 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     const bool leader = (cta_rank == 0);
     const int unit = blockIdx.x / NCTA;            // CTA or CTA pair index
     const int units = gridDim.x / NCTA;
-#ifdef FMM_TIMING
-    long long tim[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-    const long long t_kernel = clock64();
-#endif
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < C::STAGES; ++s) { mbar_init(bar_full(s), 1); mbar_init(bar_empty(s), 1); }
@@ -254,9 +242,7 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                 const int t_end = (grp + 1) * p.terms_per_group;
                 for (int t = t_end - p.terms_per_group; t < t_end && ok; ++t) {
                     for (int ks = 0; ks < kstages; ++ks) {
-                        const long long tw = TCLK();
                         if (!mbar_wait(bar_empty(stage), phase ^ 1u, ctl, 101)) { ok = false; break; }
-                        TADD(0, tw);
                         // completion is counted on the even CTA's barrier; only that CTA arms it
                         const uint32_t fb = (NCTA == 2) ? (bar_full(stage) & PEER_BIT_MASK) : bar_full(stage);
                         if (leader) mbar_expect_tx(bar_full(stage), half ? C::TX_BYTES_HALF : C::TX_BYTES);
@@ -395,15 +381,11 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                 const uint32_t idesc = half ? (idesc_full & ~(0x3Fu << 17)) | ((uint32_t)(BN >> 4) << 17) : idesc_full;
                 for (int t = 0; t < p.terms_per_group && ok; ++t) {
                     if (C::MX) {
-                        const long long tw = TCLK();
                         if (!mbar_wait(bar_tempty(0), bphase ^ 1u, ctl, 201)) { ok = false; break; }
-                        TADD(1, tw);
                         tc_fence_after();
                     }
                     for (int ks = 0; ks < kstages; ++ks) {
-                        const long long tw2 = TCLK();
                         if (!mbar_wait(bar_full(stage), phase, ctl, 202)) { ok = false; break; }
-                        TADD(2, tw2);
                         tc_fence_after();
                         const uint64_t adesc = make_kmajor_sw128_desc(base + C::OFF_A + stage * C::A_BYTES);
                         const uint64_t bdesc = make_kmajor_sw128_desc(base + C::OFF_B + stage * C::B_BYTES);
@@ -423,9 +405,7 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                         } else {
 #pragma unroll
                             for (int g0 = 0; g0 < C::KB_PER_STAGE; g0 += C::GPB) {
-                                const long long tw3 = TCLK();
                                 if (!mbar_wait(bar_tempty(buf), bphase ^ 1u, ctl, 203)) { ok = false; break; }
-                                TADD(1, tw3);
                                 tc_fence_after();
 #pragma unroll
                                 for (int gi = 0; gi < C::GPB; ++gi) {
@@ -478,9 +458,7 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             const uint32_t lane_taddr = tmem_base + ((uint32_t)(q * 32) << 16) + h * cw;
             for (int t = grp * p.terms_per_group, left = p.terms_per_group; left > 0 && ok; ++t, --left) {
                 if (C::MX) {
-                    const long long tw = TCLK();
                     if (!mbar_wait_warp(bar_tfull(0), bphase, ctl, 301)) { ok = false; break; }
-                    TADD(3, tw);
                     tc_fence_after();
 #pragma unroll
                     for (int c = 0; c < C::CW / 32; ++c)
@@ -523,9 +501,7 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                         const uint32_t sbs32 = sb_lane + ss * C::SB_STAGE_BYTES;
 #pragma unroll
                         for (int g0 = 0; g0 < C::KB_PER_STAGE; g0 += C::GPB) {
-                            const long long tw = TCLK();
                             if (!mbar_wait_warp(bar_tfull(buf), bphase, ctl, 303)) { ok = false; break; }
-                            TADD(3, tw);
                             tc_fence_after();
 #pragma unroll
                             for (int gi = 0; gi < C::GPB; ++gi) {
@@ -599,9 +575,7 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                         const uint8_t* sbs = base_ptr + C::OFF_SB + ss * C::SB_STAGE_BYTES;
 #pragma unroll
                         for (int g0 = 0; g0 < C::KB_PER_STAGE; g0 += C::GPB) {
-                            const long long tw = TCLK();
                             if (!mbar_wait_warp(bar_tfull(buf), bphase, ctl, 303)) { ok = false; break; }
-                            TADD(3, tw);
                             tc_fence_after();
 #pragma unroll
                             for (int gi = 0; gi < C::GPB; ++gi) {
@@ -646,7 +620,6 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                 if (C::DUMP) {
                     // ---- hand the finished product to the output warp: rows q*32 + lane, columns h*CW .. of the tile,
                     // as 32 x 32 chunks in the 128-byte-swizzled layout of the output tensor map
-                    const long long t_dump = TCLK();
                     if (!mbar_wait_warp(bar_dempty, dphase ^ 1u, ctl, 304)) { ok = false; break; }
                     dphase ^= 1u;
                     // thread: rows lane/4 + 8k of the warp's 32-row chunk, column pairs 8j + 2(lane%4) of its 64 columns
@@ -662,11 +635,9 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                     }
                     __syncwarp();
                     if (lane == 0) mbar_arrive(bar_dfull);
-                    TADD(4, t_dump);
                     continue;
                 }
                 // ---- post-addition: W-weighted scatter of this product into its C blocks
-                const long long t_out = TCLK();
                 // Each C tile is updated once per term that feeds it, and between two updates a whole term's operands
                 // stream through L2: the tiles are marked evict-last (at n = 8192: fewer write-backs of
                 // half-accumulated tiles, product kernel 3 % faster; evict-first on the operand loads was slower).
@@ -725,19 +696,11 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                         ++store_cnt;
                     }
                 }
-                TADD(4, t_out);
             }
         }
         if (lane == 0) bulk_wait<0>();
     }
 
-#ifdef FMM_TIMING
-    if (blockIdx.x == 0 && lane == 0 && (warp <= 1 || warp == EPI_WARP0)) {
-        long long* dst = reinterpret_cast<long long*>(p.status + 8) + (warp <= 1 ? warp : 2) * 8;
-        for (int i = 0; i < 7; ++i) dst[i] = tim[i];
-        dst[7] = clock64() - t_kernel;
-    }
-#endif
     // ---------------------------------------------------------------------- teardown
     if (*abort_flag) {
         // let copies that are still in flight towards this CTA's shared memory land

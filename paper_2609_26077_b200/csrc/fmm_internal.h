@@ -3,6 +3,7 @@
 #include <cuda_runtime.h>
 #include <cuda.h>
 #include <stdint.h>
+#include <atomic>
 #include "../../include/fmm.h"
 
 #define FMM_MAX_RANK 8
@@ -39,7 +40,9 @@ struct fmm_plan {
     int* d_out_start;         // [terms + 1]
     FmmOutEntry* d_out;       // [total entries], block offsets in units of leaf blocks (scaled at launch)
     int n_out_total;
-    int last_launches;
+    // kernels launched by the most recent call on this plan; written once, at the end of a call (calls take the
+    // plan as const, and two host threads may share one)
+    mutable std::atomic<int> last_launches;
 };
 
 struct EncodeParams {

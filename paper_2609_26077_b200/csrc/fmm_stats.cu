@@ -17,6 +17,7 @@ namespace {
 
 constexpr int STAT_BLOCKS = 592;      // 4 x 148 SMs, all resident at 512 threads; at most the 1024 slots of g_noalloc_partials
 constexpr int STAT_THREADS = 512;
+constexpr int64_t STATS_MAX_DIM = (int64_t)1 << 30;    // per dimension, as for the product itself: M * N cannot overflow
 static_assert(STAT_BLOCKS <= 1024, "one scratch slot per reduction block");
 
 __device__ __forceinline__ void warp_reduce3(double& a, double& b, double& c)
@@ -149,7 +150,8 @@ fmm_status_t fmm_error_stats(const float* C, const double* Cref, int64_t M, int6
                              void* scratch, size_t scratch_bytes, void* stream)
 {
     if (!C || !Cref || !out3 || !scratch) return FMM_ERR_INVALID_ARG;
-    if (M <= 0 || N <= 0 || ((M * N) & 1)) return FMM_ERR_SHAPE;
+    // bound each factor before forming the product (signed overflow otherwise)
+    if (M <= 0 || N <= 0 || M > STATS_MAX_DIM || N > STATS_MAX_DIM || ((M * N) & 1)) return FMM_ERR_SHAPE;
     if (scratch_bytes < fmm_error_stats_scratch_bytes() || ((uintptr_t)scratch & 15)) return FMM_ERR_WORKSPACE;
     if (((uintptr_t)C & 7) || ((uintptr_t)Cref & 15)) return FMM_ERR_INVALID_ARG;
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
@@ -173,7 +175,7 @@ fmm_status_t fmm_ref_gemm_fp64(const float* A, const float* B, double* Cref, int
 // ---- variant of fmm_error_stats for callers that cannot allocate device memory ----------------
 namespace {
 constexpr int NOALLOC_MAX_DEVICES = 64;
-constexpr int64_t NOALLOC_MAX_ELEMS = (int64_t)1 << 28;    // limit of the interface (2^18 elements per slot of the 1024-slot array)
+constexpr int64_t NOALLOC_MAX_ELEMS = (int64_t)1 << 28;    // a constant of the interface, not of the array: the kernels handle any count
 std::mutex g_noalloc_mutex;
 double* g_noalloc_ptr[NOALLOC_MAX_DEVICES] = {nullptr};
 
@@ -201,8 +203,8 @@ fmm_status_t fmm_error_stats_noalloc(const float* C, const double* Cref, int64_t
                                      void* stream)
 {
     if (!C || !Cref || !out3) return FMM_ERR_INVALID_ARG;
-    if (M <= 0 || N <= 0 || ((M * N) & 1)) return FMM_ERR_SHAPE;
-    if (M > NOALLOC_MAX_ELEMS || N > NOALLOC_MAX_ELEMS || M * N > NOALLOC_MAX_ELEMS) return FMM_ERR_SHAPE;
+    if (M <= 0 || N <= 0 || M > NOALLOC_MAX_ELEMS || N > NOALLOC_MAX_ELEMS) return FMM_ERR_SHAPE;
+    if (M * N > NOALLOC_MAX_ELEMS || ((M * N) & 1)) return FMM_ERR_SHAPE;
     if (((uintptr_t)C & 7) || ((uintptr_t)Cref & 15)) return FMM_ERR_INVALID_ARG;
     double* partial = nullptr;
     fmm_status_t s = noalloc_scratch(&partial);

@@ -8,11 +8,11 @@ import os
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.environ.get("FMM_B200_LIB", os.path.join(_HERE, "libfmm_b200.so"))   # override: experiment builds
+LIB_PATH = os.path.join(_HERE, "libfmm_b200.so")
 
 FMM_OK = 0
 STATUS_NAMES = ["FMM_OK", "FMM_ERR_INVALID_ARG", "FMM_ERR_SHAPE", "FMM_ERR_NOT_EXACT", "FMM_ERR_WORKSPACE",
-                "FMM_ERR_ALLOC", "FMM_ERR_CUDA", "FMM_ERR_ARCH", "FMM_ERR_DEVICE_TIMEOUT"]
+                "FMM_ERR_ALLOC", "FMM_ERR_CUDA", "FMM_ERR_ARCH", "FMM_ERR_DEVICE_TIMEOUT", "FMM_ERR_WRONG_DEVICE"]
 SCALE_FP32, SCALE_UE8M0 = 0, 1
 SCALE_MODES = {"fp32": SCALE_FP32, "ue8m0": SCALE_UE8M0}
 

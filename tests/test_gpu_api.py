@@ -174,3 +174,33 @@ def test_host_operand_call_rejects_bad_arguments():
     assert call(256, p(ws), ws.numel(), A=None) == 1
     need = C.c_size_t()
     assert lib.fmm_host_workspace_bytes(plan._h, C.c_int64(100), C.c_int64(256), C.c_int64(256), C.byref(need)) == 2
+    assert lib.fmm_host_workspace_bytes(plan._h, C.c_int64(256), C.c_int64(256), C.c_int64(256), None) == 1
+    assert lib.fmm_host_workspace_bytes(None, C.c_int64(256), C.c_int64(256), C.c_int64(256), C.byref(need)) == 1
+
+
+def test_status_is_read_after_work_on_a_non_blocking_stream():
+    # fmm_device_status waits for every stream of the device, also streams that do not synchronise with the
+    # default stream (torch's side streams are of that kind): the timeout set by a kernel still running there is seen
+    plan = make_plan("strassen", 1, 32, "ue8m0")
+    side = torch.cuda.Stream()
+    assert fmm.lib().fmm_selftest_bounded_wait(plan._h, C.c_int64(50_000_000), C.c_void_p(side.cuda_stream)) == 0
+    assert plan.device_status() == (8, 901)             # read right away, no explicit synchronisation
+    plan.device_status_clear()
+    assert plan.device_status() == (0, 0)
+    plan.close()
+
+
+@pytest.mark.skipif(torch.cuda.device_count() < 2, reason="needs two devices")
+def test_call_on_another_device_is_refused():
+    plan = make_plan("strassen", 1, 32, "ue8m0")
+    ws = plan.workspace(256, 256, 256)
+    a = torch.zeros(256, 256, device="cuda:0")
+    torch.cuda.set_device(1)
+    try:
+        rc = fmm.lib().fmm_matmul(plan._h, C.c_void_p(a.data_ptr()), C.c_void_p(a.data_ptr()), C.c_void_p(a.data_ptr()),
+                                  C.c_int64(256), C.c_int64(256), C.c_int64(256), C.c_void_p(ws.data_ptr()),
+                                  C.c_size_t(ws.numel()), None)
+        assert rc == 9
+    finally:
+        torch.cuda.set_device(0)
+    plan.close()

@@ -1,6 +1,7 @@
 """GPU parity at the benchmark's full size (n = 8192, one level, Phi-optimal: the launch configuration
 bench.py times).  The quantized operands are compared in full against the oracle; C is compared on
-sampled rows that the oracle side computes one by one from its own quantized operands."""
+sampled rows and on sampled 128 x 128 tiles of every output block, which the oracle's own C code computes
+entry by entry from its own quantized operands (plain loops, fp64)."""
 import numpy as np
 import pytest
 import torch
@@ -27,24 +28,32 @@ def test_full_size_operands_bit_exact_and_sampled_rows_of_c(mode, blk):
     cb, sb, eb = O.encode(B, "B", U, V, 1, blk, MODES[mode])
     rng = np.random.default_rng(1)
     rows = np.sort(rng.choice(h, size=24, replace=False))
-    Mrows = []
+    # four 128 x 128 tiles of the leaf index space (each is compared in all four output blocks), not aligned to the
+    # kernel's 256-row / 256-column tile positions
+    tiles = [(int(r), int(c)) for r, c in zip(rng.integers(0, h - 128, 4), rng.integers(0, h - 128, 4))]
+    allcols = np.arange(h)
+    Mrows, Mtiles = [], []
     for t in range(7):
         qa, sca = plan.quantized_operand(ws, n, n, n, t, "A")
         qb, scb = plan.quantized_operand(ws, n, n, n, t, "B")
         assert np.array_equal(qa, ca[t]) and np.array_equal(qb, cb[t]), f"codes differ in term {t}"
         assert np.array_equal(sca, sa[t] if mode == "fp32" else ea[t]), f"A scales differ in term {t}"
         assert np.array_equal(scb, sb[t] if mode == "fp32" else eb[t]), f"B scales differ in term {t}"
-        # oracle side of the product for the sampled rows: exact dequantization, fp64 matmul
-        Sr = O.dequant_rows(ca[t][rows], sa[t][rows], blk)
-        Tr = O.dequant_cols(cb[t], sb[t], blk)
-        Mrows.append(Sr @ Tr)
+        Mrows.append(O.leaf_product_sample(ca[t], sa[t], cb[t], sb[t], blk, rows, allcols))
+        Mtiles.append([O.leaf_product_sample(ca[t], sa[t], cb[t], sb[t], blk, np.arange(r, r + 128), np.arange(c, c + 128))
+                       for r, c in tiles])
     got = C.cpu().numpy().astype(np.float64)
     for q in range(4):
-        want = sum(float(W[r][q]) * Mrows[r] for r in range(7))
         r0, c0 = (q >> 1) * h, (q & 1) * h
+        want = sum(float(W[r][q]) * Mrows[r] for r in range(7))
         block = got[r0 + rows][:, c0:c0 + h]
         rel = np.linalg.norm(block - want) / np.linalg.norm(want)
         assert rel <= 1e-5, f"quadrant {q}: sampled rows differ by {rel:.3e}"
+        for i, (tr, tc) in enumerate(tiles):
+            want = sum(float(W[r][q]) * Mtiles[r][i] for r in range(7))
+            tile = got[r0 + tr:r0 + tr + 128, c0 + tc:c0 + tc + 128]
+            rel = np.linalg.norm(tile - want) / np.linalg.norm(want)
+            assert rel <= 1e-5, f"quadrant {q}, tile at ({tr},{tc}): differs by {rel:.3e}"
     assert np.isfinite(got).all()
 
 
@@ -71,7 +80,7 @@ def test_full_size_two_levels_operands_bit_exact_and_sampled_rows_of_c():
         qb, scb = plan.quantized_operand(ws, n, n, n, t, "B")
         assert np.array_equal(qa, ca[t]) and np.array_equal(qb, cb[t]), f"codes differ in term {t}"
         assert np.array_equal(sca, ea[t]) and np.array_equal(scb, eb[t]), f"scales differ in term {t}"
-        Mrows.append(O.dequant_rows(ca[t][rows], sa[t][rows], blk) @ O.dequant_cols(cb[t], sb[t], blk))
+        Mrows.append(O.leaf_product_sample(ca[t], sa[t], cb[t], sb[t], blk, rows, np.arange(leaf)))
     got = C.cpu().numpy().astype(np.float64)
     assert np.isfinite(got).all()
     for q1 in range(4):
@@ -106,7 +115,7 @@ def test_full_size_rectangular_llm_shape_sampled_rows_of_c():
         qb, scb = plan.quantized_operand(ws, M, N, K, t, "B")
         assert np.array_equal(qa, ca[t]) and np.array_equal(qb, cb[t]), f"codes differ in term {t}"
         assert np.array_equal(sca, sa[t]) and np.array_equal(scb, sb[t]), f"scales differ in term {t}"
-        Mrows.append(O.dequant_rows(ca[t][rows], sa[t][rows], blk) @ O.dequant_cols(cb[t], sb[t], blk))
+        Mrows.append(O.leaf_product_sample(ca[t], sa[t], cb[t], sb[t], blk, rows, np.arange(N // 2)))
     got = C.cpu().numpy().astype(np.float64)
     assert np.isfinite(got).all()
     for q in range(4):

@@ -109,6 +109,24 @@ def test_fused_result_is_decoded_sum_of_leaf_products(levels):
     assert np.allclose(got, want, rtol=1e-12, atol=1e-12)
 
 
+@pytest.mark.parametrize("mode,blk", [(O.SCALE_FP32, 32), (O.SCALE_UE8M0, 32), (O.SCALE_FP32, 128)])
+def test_sampled_leaf_product_equals_entries_of_the_whole_product(mode, blk):
+    # the sampled-entry routine used at full size: its entries are those of the cubic fp8 product (one leaf),
+    # bit for bit (same dequantization, same summation order), and a brute-force sum in Python agrees
+    A, B = Wl.gaussian(96, 128, 256, 7)
+    ca, sa, _ = O.quant_rows(A, blk, mode)
+    cb, sb, _ = O.quant_cols(B, blk, mode)
+    rows, cols = [0, 5, 17, 95], [3, 64, 65, 127, 8]
+    got = O.leaf_product_sample(ca, sa, cb, sb, blk, rows, cols)
+    whole = O.fused_fmm(A, B, levels=0, blk=blk, mode=mode)
+    assert np.array_equal(got, whole[np.ix_(rows, cols)])
+    da, db = O.dequant_rows(ca, sa, blk), O.dequant_cols(cb, sb, blk)
+    brute = brute_force(da[rows], db[:, cols])
+    assert np.allclose(got, brute, rtol=1e-14, atol=1e-14)
+    # a transposed or shifted index would be caught: entries of different rows / columns differ
+    assert not np.allclose(got[0], got[1]) and not np.allclose(got[:, 0], got[:, 1])
+
+
 def _mean_errors(family, n, blk, levels, seeds, names=("cubic", "strassen", "winograd", "phi_optimal"),
                  mode=O.SCALE_FP32):
     out = {k: [] for k in names}

@@ -162,3 +162,33 @@ def test_winograd_rebalance_factors():
     s = [math.sqrt(math.sqrt(float(R.sqnorm(U[r])) / float(R.sqnorm(V[r])))) for r in range(7)]
     off = sorted(x for x in s if abs(x - 1) > 1e-12)
     assert off == pytest.approx([1 / math.sqrt(2), math.sqrt(2)])
+
+
+def test_second_order_form_and_hessian_spectrum_at_the_optimum():
+    # App. A, second-order form: Phi_t = 200/9 + (8/9) t^T diag(Q, Q) t + O(|t|^3) with the printed Q; the
+    # coordinate Hessian has eigenvalues 128/9 (twice) and 440/9 (four times).  All in exact arithmetic.
+    U, V, W = R.phi_optimal()
+    Qm = [[Fr(21), Fr(-13, 2), Fr(-13, 2)], [Fr(-13, 2), Fr(21), Fr(-13, 2)], [Fr(-13, 2), Fr(-13, 2), Fr(21)]]
+    Hs = R.phi_hessian(U, V, W)
+    for i in range(6):
+        for j in range(6):
+            same_block = (i // 3) == (j // 3)
+            want = Fr(16, 9) * Qm[i % 3][j % 3] if same_block else Fr(0)
+            assert Hs[i][j] == Q3(want), (i, j, Hs[i][j])
+    # stationarity (zero moment map): no first-order term in any coordinate or pair direction
+    for d in ([1, 0, 0, 0, 0, 0], [0, 0, 0, 0, 1, 0], [1, -2, 3, 5, -1, 2]):
+        c0, c1, _ = R.phi_second_order(U, V, W, d)
+        assert c0 == Q3(Fr(200, 9)) and c1.is_zero()
+    # spectrum: (H - 128/9)(H - 440/9) = 0 with trace 2 * 128/9 + 4 * 440/9, so exactly those multiplicities
+    lo, hi = Fr(128, 9), Fr(440, 9)
+    Hf = [[Hs[i][j].a for j in range(6)] for i in range(6)]
+    A1 = [[Hf[i][j] - (lo if i == j else 0) for j in range(6)] for i in range(6)]
+    A2 = [[Hf[i][j] - (hi if i == j else 0) for j in range(6)] for i in range(6)]
+    prod = [[sum(A1[i][k] * A2[k][j] for k in range(6)) for j in range(6)] for i in range(6)]
+    assert all(x == 0 for row in prod for x in row)
+    assert sum(Hf[i][i] for i in range(6)) == 2 * lo + 4 * hi
+    assert np.allclose(np.sort(np.linalg.eigvalsh(np.array(Hf, dtype=float))),
+                       [128 / 9] * 2 + [440 / 9] * 4, rtol=1e-12)
+    # control: classic Strassen is not a stationary point of Phi on its orbit
+    c0, c1, _ = R.phi_second_order(*R.strassen(), [0, 0, 0, 1, 0, 0])
+    assert c0 == Q3(32) and not c1.is_zero()
