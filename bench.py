@@ -45,8 +45,8 @@ def parse():
     ap.add_argument("--scale-mode", default="fp32", choices=["fp32", "ue8m0"])
     ap.add_argument("--block-k", type=int, default=32, choices=[32, 128])
     ap.add_argument("--no-variants", action="store_true")
-    ap.add_argument("--ref-n", type=int, default=1024, help="sample size of one reference (oracle) step")
-    ap.add_argument("--cpu-baseline-n", type=int, default=0, help="0 = 4096 with >= 8 host threads, else 2048")
+    ap.add_argument("--ref-n", type=int, default=0, help="reference arm: size of one oracle step (0 = --n / 2, --n / 4 with few host threads)")
+    ap.add_argument("--cpu-baseline-n", type=int, default=0, help="size of the oracle pass of the cpu_baseline leg (0 = --n)")
     return ap.parse_args()
 
 
@@ -139,18 +139,37 @@ def algorithmic_work(M, N, K, levels, rank, scale_bytes, blk):
     return flops, enc_bytes, gemm_bytes
 
 
+SPEC_FP8_TFLOPS, SPEC_HBM_GBS = 4500.0, 8000.0      # B200 nominal dense fp8 and HBM3e figures
+
+
 def combined_roofline_ms(M, N, K, levels, rank, mode, blk, fp8_peak_tflops, hbm_gbs):
-    """Combined roofline time of one pass: the product phase at the measured fp8 tensor peak - or, with fp32 scales, at
-    the CUDA-core bound of the per-block promotion if that is larger - plus the algorithmic HBM bytes at the measured
-    copy bandwidth (phases serialized)."""
-    scale_bytes = 1 if mode == "ue8m0" else 4
+    """Combined roofline time of one pass: the product phase at the fp8 tensor peak plus the algorithmic HBM bytes
+    (pre-addition + quantization, operand reads of the products, one write of C) at the copy bandwidth, phases
+    serialized.  The same formula for every scale mode."""
+    scale_bytes = 1 if mode.startswith("ue8m0") else 4
     flops, enc_bytes, gemm_bytes = algorithmic_work(M, N, K, levels, rank, scale_bytes, blk)
-    t_main = flops / (fp8_peak_tflops * 1e12)
-    if mode != "ue8m0":
-        f = (rank / 8.0) ** levels if levels > 0 else 1.0
-        ops = 1.0 if "tile" in mode else 2.0        # weight tiles: the factor is formed once per row, one FMA per element
-        t_main = max(t_main, ops * M * N * (K / blk) * f / (148 * 128 * 1.965e9))
-    return (t_main + (enc_bytes + gemm_bytes) / (hbm_gbs * 1e9)) * 1e3
+    return (flops / (fp8_peak_tflops * 1e12) + (enc_bytes + gemm_bytes) / (hbm_gbs * 1e9)) * 1e3
+
+
+def alu_floor_ms(M, N, K, levels, rank, mode, blk):
+    """fp32 scales only: CUDA-core time of the per-block promotion acc += P * (sA * sB) that the chosen algorithm
+    needs (the tensor core cannot apply a per-row x per-column fp32 factor per K block): M*N*(K/blk) elements,
+    1 mul + 1 fma each (1 fma with 128 x 128 weight tiles), on 148 SMs x 128 fp32 lanes at the 1.965 GHz maximum
+    clock.  A floor of this implementation's design, reported beside the roofline and not part of it."""
+    if mode.startswith("ue8m0"):
+        return 0.0
+    f = (rank / 8.0) ** levels if levels > 0 else 1.0
+    ops = 1.0 if "tile" in mode else 2.0
+    return ops * M * N * (K / blk) * f / (148 * 128 * 1.965e9) * 1e3
+
+
+def roofline_fractions(M, N, K, levels, rank, mode, blk, ms, pk):
+    """Fractions of the combined roofline against the measured and the nominal peaks, plus the ALU floor."""
+    meas = combined_roofline_ms(M, N, K, levels, rank, mode, blk, 2.0 * pk["bf16_tflops"], pk["hbm_gbs"])
+    spec = combined_roofline_ms(M, N, K, levels, rank, mode, blk, SPEC_FP8_TFLOPS, SPEC_HBM_GBS)
+    return {"combined_roofline_ms": meas, "combined_frac": meas / ms,
+            "combined_roofline_spec_ms": spec, "combined_frac_spec": spec / ms,
+            "alu_floor_ms": alu_floor_ms(M, N, K, levels, rank, mode, blk)}
 
 
 def run_ours(args):
@@ -283,7 +302,7 @@ def run_ours(args):
         "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "fp8_e4m3", "data": "synthetic",
         "config": {"workload": (f"n={n} square" if not args.shape else f"M,K,N={M},{K},{N}") +
-                               f", {args.levels} level(s), {args.realization}, A,B iid N(0,1) fp32 (BASELINE configs[2])",
+                               f", {args.levels} level(s), {args.realization}, A,B iid N(0,1) fp32",
                    "scale_mode": args.scale_mode, "block_k": args.block_k, "M": M, "N": N, "K": K,
                    "l2": f"inputs larger than L2 ({4 * M * K / 1e6:.0f} + {4 * K * N / 1e6:.0f} MB fp32 operands, {4 * M * N / 1e6:.0f} MB output)",
                    "multi_gpu": "replicas only"},
@@ -299,35 +318,26 @@ def run_ours(args):
                    "multiply_tflops": flops_alg / (mul_ms * 1e-3) / 1e12},
         "device_status": status[1],
     }
-    # dominant kernel = the tcgen05 product kernel.  DRAM traffic per launch: dram__bytes_read + write from one-pass
-    # ncu captures of this command (profiles/fmm_gemm_kernel_dram_traffic.md).  At n = 8192 the live C tiles and the
-    # operand streams no longer fit L2 together, so traffic does not scale with M*N: only measured sizes are reported.
+    # dominant kernel = the tcgen05 product kernel, timed live above (events around fmm_multiply_only).
+    # DRAM traffic per launch comes from one-pass ncu captures of this command (two counters); the live C tiles and
+    # the operand streams compete for L2, so traffic does not scale with M*N and only captured sizes are reported.
     measured = {("fp32", 32, 8192): 1521.0e6, ("ue8m0", 32, 8192): 1623.0e6,
                 ("fp32", 32, 4096): 136.4e6, ("ue8m0", 32, 4096): 151.0e6}
     traffic = None
     if args.levels == 1 and M == N == K and args.realization == "phi_optimal":
         traffic = measured.get((args.scale_mode, args.block_k, M))
-    t_roof_ms = (flops_alg / (fp8_peak * 1e12) + (enc_bytes + gemm_bytes) / (hbm * 1e9)) * 1e3
+    mode_name = args.scale_mode
     out["roofline"] = {"kernel": "fmm_gemm_kernel", "bound": "tensor",
                        "achieved": flops_alg / (mul_ms * 1e-3) / 1e12, "peak": fp8_peak, "unit": "TFLOP/s",
-                       "frac": flops_alg / (mul_ms * 1e-3) / 1e12 / fp8_peak, "traffic": traffic,
-                       "traffic_unit": "bytes per launch (ncu dram__bytes_read.sum + dram__bytes_write.sum at this size)", "algorithmic_bytes": gemm_bytes,
-                       "peak_source": f"2 x {pk['source']} bf16 burst ({pk['bf16_tflops']} TF/s)",
-                       "combined_roofline_ms": t_roof_ms, "combined_frac": t_roof_ms / ms_step}
-    if args.scale_mode == "fp32":
-        # the per-block fp32 x fp32 scale promotion runs on the CUDA cores: M*N*(K/blk) x (1 mul + 1 fma) lane-ops
-        f = (rank_r / 8.0) ** args.levels if args.levels > 0 else 1.0
-        lane_ops = 2.0 * M * N * (K / args.block_k) * f
-        alu_peak = 148 * 128 * 1.965e9              # fp32 lanes x max SM clock, one op per lane per clock
-        t_alu, t_tc = lane_ops / alu_peak, flops_alg / (fp8_peak * 1e12)
-        t_roof_ms = (max(t_alu, t_tc) + (enc_bytes + gemm_bytes) / (hbm * 1e9)) * 1e3
-        r = out["roofline"]
-        r.update({"tensor_achieved_tflops": r["achieved"], "tensor_frac": r["frac"],
-                  "combined_roofline_ms": t_roof_ms, "combined_frac": t_roof_ms / ms_step})
-        if t_alu > t_tc:
-            r.update({"bound": "alu", "achieved": lane_ops / (mul_ms * 1e-3) / 1e12, "peak": alu_peak / 1e12,
-                      "unit": "T fp32 lane-op/s", "frac": lane_ops / (mul_ms * 1e-3) / alu_peak,
-                      "peak_source": "148 SMs x 128 fp32 lanes x 1.965 GHz (unit counts and max clock)"})
+                       "frac": flops_alg / (mul_ms * 1e-3) / 1e12 / fp8_peak,
+                       "frac_spec": flops_alg / (mul_ms * 1e-3) / 1e12 / SPEC_FP8_TFLOPS,
+                       "traffic": traffic,
+                       "traffic_source": ("ncu dram__bytes_read.sum + dram__bytes_write.sum, one-pass capture of this "
+                                          "command at this size" if traffic else None),
+                       "algorithmic_bytes": gemm_bytes,
+                       "peak_source": f"2 x {pk['source']} bf16 burst ({pk['bf16_tflops']} TF/s); spec {SPEC_FP8_TFLOPS} TF/s, {SPEC_HBM_GBS} GB/s",
+                       "hbm_peak_gbs": hbm}
+    out["roofline"].update(roofline_fractions(M, N, K, args.levels, rank_r, mode_name, args.block_k, ms_step, pk))
 
     if rank_id == 0 and world == 1 and not args.no_variants:
         variants = []
@@ -344,12 +354,41 @@ def run_ours(args):
             p2 = make_plan(name, lv, blk, mode)
             w2 = p2.workspace(M, N, K)
             ms = time_steps(lambda: p2.matmul(A, B, out=C, workspace=w2), 5, 3)
-            t_roof = combined_roofline_ms(M, N, K, lv, p2.rank if lv > 0 else 8, mode, blk, fp8_peak, hbm)
-            variants.append({"realization": name, "levels": lv, "block_k": blk, "scale_mode": mode,
-                             "ms_per_step": ms, "value": flop_eff / (ms * 1e-3) / 1e12,
-                             "combined_roofline_ms": t_roof, "combined_frac": t_roof / ms})
+            v = {"realization": name, "levels": lv, "block_k": blk, "scale_mode": mode,
+                 "ms_per_step": ms, "value": flop_eff / (ms * 1e-3) / 1e12}
+            v.update(roofline_fractions(M, N, K, lv, p2.rank if lv > 0 else 8, mode, blk, ms, pk))
+            if lv >= 2:
+                # outside the algorithmic bytes: the outer decoder reads the 7 partially decoded products of every
+                # parent and writes its four blocks (its own kernel, one extra HBM round trip per outer level)
+                v["decode_round_trip_bytes"] = sum(4.0 * M * N * ((7.0 / 4.0) ** l + (7.0 / 4.0) ** (l - 1)) for l in range(1, lv))
+            variants.append(v)
             p2.close()
         out["variants"] = variants
+        # rectangular LLM-shaped case: M, K, N = 16384, 8192, 8192, A = N(0,1) rows with per-column lognormal(0, 1.5)
+        # outlier channels, B ~ N(0, 0.02^2); rank-7 at one level next to the cubic product in the same kernels
+        if M == N == K == 8192 and args.levels == 1:
+            Mr, Kr, Nr = 16384, 8192, 8192
+            Ar = torch.randn(Mr, Kr, device="cuda", generator=gen) * torch.exp(1.5 * torch.randn(Kr, device="cuda", generator=gen))
+            Br = 0.02 * torch.randn(Kr, Nr, device="cuda", generator=gen)
+            Cr = torch.empty(Mr, Nr, device="cuda")
+            rect = []
+            for name, lv, blk, mode in [("phi_optimal", 1, args.block_k, args.scale_mode), ("strassen", 1, args.block_k, args.scale_mode),
+                                        ("cubic", 0, args.block_k, args.scale_mode),
+                                        ("phi_optimal", 1, 128, "fp32"), ("cubic", 0, 128, "fp32"),
+                                        ("phi_optimal", 1, 32, "ue8m0"), ("strassen", 1, 32, "ue8m0"), ("cubic", 0, 32, "ue8m0")]:
+                p2 = make_plan(name, lv, blk, mode)
+                w2 = p2.workspace(Mr, Nr, Kr)
+                ms = time_steps(lambda: p2.matmul(Ar, Br, out=Cr, workspace=w2), 5, 3)
+                v = {"realization": name, "levels": lv, "block_k": blk, "scale_mode": mode, "ms_per_step": ms,
+                     "value": 2.0 * Mr * Nr * Kr / (ms * 1e-3) / 1e12}
+                v.update(roofline_fractions(Mr, Nr, Kr, lv, p2.rank if lv > 0 else 8, mode, blk, ms, pk))
+                rect.append(v)
+                p2.close()
+                del w2
+            out["rectangular"] = {"workload": f"M,K,N={Mr},{Kr},{Nr}, A rows N(0,1) x per-column lognormal(0,1.5) factors, B iid N(0,0.02)",
+                                  "arms": rect}
+            del Ar, Br, Cr
+            torch.cuda.empty_cache()
         # the paper's timing protocol (App. E.7): interleaved repetitions across realizations, median and a
         # bootstrap 95 % interval of the median, so that clock drift hits every arm alike
         arms = [("cubic", 0), ("strassen", 1), ("phi_optimal", 1)]
@@ -397,8 +436,7 @@ def run_ours(args):
             "error_stats": {"ms": ms_stats, "gbs": 12.0 * M * N / (ms_stats * 1e-3) / 1e9,
                             "hbm_frac": 12.0 * M * N / (ms_stats * 1e-3) / 1e9 / hbm, "bytes": 12.0 * M * N},
             "ref_gemm_fp64": {"ms": ms_ref, "tflops_fp64": 2.0 * M * N * K / (ms_ref * 1e-3) / 1e12}}
-        from oracle import oracle as _O
-        out["cpu_baseline"] = cpu_baseline(args, args.cpu_baseline_n or (4096 if _O.num_threads() >= 8 else 2048))
+        out["cpu_baseline"] = cpu_baseline(args)
     elif rank_id == 0:
         out["cpu_baseline"] = None
 
@@ -411,6 +449,7 @@ def run_ours(args):
 
 # ------------------------------------------------------------------------------------------------
 def _oracle_step(n, levels, realization, blk, mode, seed=0):
+    """One oracle pass over an n x n x n problem of the benchmarked kind; returns the seconds it took."""
     import numpy as np
     from oracle import oracle as O, realizations as R
     from paper_2609_26077_b200 import workloads as Wl
@@ -422,31 +461,38 @@ def _oracle_step(n, levels, realization, blk, mode, seed=0):
     return time.perf_counter() - t0
 
 
-def cpu_baseline(args, n):
+def cpu_baseline(args):
+    """The oracle as it stands, timed once on the benchmarked configuration itself (n = 8192: about half a minute on
+    16 cores); with fewer than 8 host threads one pass at half the size is timed instead and the sample says so."""
     from oracle import oracle as O
+    n = args.cpu_baseline_n or (args.n if O.num_threads() >= 8 else args.n // 2)
     t = _oracle_step(n, args.levels, args.realization, args.block_k, args.scale_mode)
-    return {"value": 2.0 * n ** 3 / t / 1e12, "unit": UNIT, "cores": O.num_threads(), "kind": "oracle",
-            "seconds": t, "sample": f"one oracle pass of the same path at n={n} (same realization, levels, quantizer), "
-                                    f"scaled by 2n^3/t; the full n={args.n} case costs (n/{n})^3 more"}
+    what = "the benchmarked size" if n == args.n else f"a smaller instance of the n={args.n} workload (its cost grows as n^3)"
+    return {"value": 2.0 * n ** 3 / t / 1e12, "unit": UNIT, "cores": O.num_threads(), "kind": "oracle", "seconds": t,
+            "sample": f"one oracle pass at n={n}, {what} (same realization, levels, quantizer); value = 2n^3/t"}
 
 
 def run_reference(args):
     if int(os.environ.get("RANK", "0")) != 0:
         return
     from oracle import oracle as O
-    n = args.ref_n
+    # bounded sample: one step = one oracle pass at half the benchmarked size (an eighth of the work; about 4 s on 16
+    # cores at n = 4096, so that warm-up plus 20 steps end within a few minutes), a quarter with few host threads
+    n = args.ref_n or (args.n // 2 if O.num_threads() >= 8 else args.n // 4)
     for _ in range(args.warmup):
         _oracle_step(n, args.levels, args.realization, args.block_k, args.scale_mode)
     ts = [_oracle_step(n, args.levels, args.realization, args.block_k, args.scale_mode, seed=i)
           for i in range(args.steps)]
     t = sum(ts) / len(ts)
     val = 2.0 * n ** 3 / t / 1e12
-    sample = f"each step = one oracle pass at n={n} (bounded sample of the n={args.n} workload), value = 2n^3/t"
+    sample = (f"each step = one oracle pass at n={n} (bounded sample of the n={args.n} workload: same realization, levels, "
+              f"quantizer and operand family, smaller matrices), value = 2n^3/t")
     out = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
            "steps": args.steps, "warmup": args.warmup, "ms_per_step": t * 1e3, "higher_is_better": True,
            "scaling": "weak", "vs_baseline": None, "dtype": "fp8_e4m3", "data": "synthetic",
-           "config": {"workload": f"n={args.n} square, {args.levels} level(s), {args.realization}, A,B iid N(0,1) fp32 (BASELINE configs[2])",
-                      "scale_mode": args.scale_mode, "block_k": args.block_k, "sample_n": n},
+           "config": {"workload": f"n={args.n} square, {args.levels} level(s), {args.realization}, A,B iid N(0,1) fp32",
+                      "scale_mode": args.scale_mode, "block_k": args.block_k, "M": args.n, "N": args.n, "K": args.n,
+                      "l2": "not applicable (host cores)", "multi_gpu": "replicas only", "sample_n": n},
            "cpu_baseline": {"value": val, "unit": UNIT, "cores": O.num_threads(), "kind": "oracle", "sample": sample},
            "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
            "gpu_launches": 0}

@@ -54,21 +54,24 @@ def test_algorithmic_work_matches_the_derivation():
 
 
 def test_combined_roofline_time_follows_the_derivation():
-    # n = 8192, one level: tensor phase at the given fp8 peak, or the fp32 promotion bound (2 lane-ops per element
-    # and 32-k block on 148 x 128 lanes at 1.965 GHz) if larger, plus the algorithmic bytes at the given bandwidth
+    # n = 8192, one level: tensor phase at the given fp8 peak plus the algorithmic bytes at the given bandwidth,
+    # the same formula in every scale mode; 380.5 us at the nominal peaks (4.5 PFLOP/s, 8 TB/s)
     n, peak, bw = 8192, 3293.6, 6459.0
-    flops, enc, gemm = bench.algorithmic_work(n, n, n, 1, 7, 1, 32)
-    want = (flops / (peak * 1e12) + (enc + gemm) / (bw * 1e9)) * 1e3
-    assert bench.combined_roofline_ms(n, n, n, 1, 7, "ue8m0", 32, peak, bw) == pytest.approx(want, rel=1e-12)
-    flops, enc, gemm = bench.algorithmic_work(n, n, n, 1, 7, 4, 32)
-    alu = 2.0 * n * n * (n / 32) * (7 / 8) / (148 * 128 * 1.965e9)
-    assert alu > flops / (peak * 1e12)
-    want = (alu + (enc + gemm) / (bw * 1e9)) * 1e3
-    assert bench.combined_roofline_ms(n, n, n, 1, 7, "fp32", 32, peak, bw) == pytest.approx(want, rel=1e-12)
-    # weight tiles: one FMA per element and 128-k block, so the tensor phase is the larger term again
-    t = bench.combined_roofline_ms(n, n, n, 1, 7, "fp32+tile128", 128, peak, bw)
-    flops, enc, gemm = bench.algorithmic_work(n, n, n, 1, 7, 4, 128)
-    assert t == pytest.approx((flops / (peak * 1e12) + (enc + gemm) / (bw * 1e9)) * 1e3, rel=1e-12)
+    for mode, sbytes, blk in (("ue8m0", 1, 32), ("fp32", 4, 32), ("fp32", 4, 128), ("fp32+tile128", 4, 128)):
+        flops, enc, gemm = bench.algorithmic_work(n, n, n, 1, 7, sbytes, blk)
+        want = (flops / (peak * 1e12) + (enc + gemm) / (bw * 1e9)) * 1e3
+        assert bench.combined_roofline_ms(n, n, n, 1, 7, mode, blk, peak, bw) == pytest.approx(want, rel=1e-12)
+    spec = bench.combined_roofline_ms(n, n, n, 1, 7, "fp32", 32, bench.SPEC_FP8_TFLOPS, bench.SPEC_HBM_GBS)
+    assert spec == pytest.approx(0.3805, rel=2e-3)
+    assert bench.combined_roofline_ms(n, n, n, 1, 7, "fp32", 32, peak, bw) == pytest.approx(0.4986, rel=2e-3)
+    # the CUDA-core floor of the fp32-scale promotion is reported beside the roofline, never inside it
+    alu = 2.0 * n * n * (n / 32) * (7 / 8) / (148 * 128 * 1.965e9) * 1e3
+    assert bench.alu_floor_ms(n, n, n, 1, 7, "fp32", 32) == pytest.approx(alu, rel=1e-12)
+    assert bench.alu_floor_ms(n, n, n, 1, 7, "fp32+tile128", 128) == pytest.approx(alu / 8, rel=1e-12)
+    assert bench.alu_floor_ms(n, n, n, 1, 7, "ue8m0", 32) == 0.0
+    pk = {"bf16_tflops": 1646.8, "hbm_gbs": 6459.0}
+    fr = bench.roofline_fractions(n, n, n, 1, 7, "fp32", 32, 2.0385, pk)
+    assert fr["combined_frac"] == pytest.approx(0.245, abs=2e-3) and fr["combined_frac_spec"] == pytest.approx(0.187, abs=2e-3)
 
 
 def test_reference_arm_prints_one_json_line():
