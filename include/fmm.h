@@ -142,8 +142,10 @@ fmm_status_t fmm_multiply_only(const fmm_plan_t* plan, float* C, int64_t M, int6
  * r1 = outermost level; 0 for levels == 0) lives in the workspace (host call, byte offsets).
  *   side 'A': codes are q_rows x q_cols = (M/d) x (K/d) e4m3 bytes, row-major (K contiguous).
  *   side 'B': codes are stored TRANSPOSED, q_rows x q_cols = (N/d) x (K/d) (K contiguous).
- *   FP32 scale mode: fp32 scales; side 'A': scale_rows x scale_cols = (M/d) x (K/d/block_k) row-major;
- *             side 'B': (K/d/block_k) x (N/d) row-major.
+ *   FP32 scale mode: fp32 scales, laid out as the product kernel fetches them per 128-k pipeline stage.
+ *             side 'A': chunk-major, [c][i][g] = scale of K block c * (128/block_k) + g of row i, with c the 128-k
+ *             chunk; reported as scale_rows x scale_cols = (K/d/128) x ((M/d) * (128/block_k)) row-major;
+ *             side 'B': (K/d/block_k) x (N/d) row-major, entry [kb][j] = scale of block kb of column j.
  *   UE8M0 mode: one biased-exponent byte per block in 512-byte tiles of 128 rows x 4 blocks:
  *             tile index (block/4) * (rows/128) + (row/128), byte (row%32)*16 + ((row%128)/32)*4 + block%4
  *             where row is the M/d (side 'A') or N/d (side 'B') index; scale_rows x scale_cols then

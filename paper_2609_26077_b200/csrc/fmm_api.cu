@@ -139,16 +139,14 @@ fmm_status_t encode_side(const fmm_plan* plan, const FmmLayout& L, char* ws, con
             } else {
                 e.rows = (int)(rows / 4); e.cols = (int)cols;
                 for (int j = 0; j < 4; ++j) e.qoff[j] = (int64_t)j * (rows / 4) * cols;
-                e.s_step = (int)(rows / 4); e.s_ld = 0; e.sf_blocks = (int)(rows / 128);
+                e.s_step = (int)(rows / 4); e.s_ld = (int)rows; e.sf_blocks = (int)(rows / 128);
             }
-            // fp32 scales of the A side and all codes are contiguous per panel; shared arrays otherwise
-            const bool fp32 = mode == FMM_SCALE_FP32_AMAX_DIV_448;
-            if (!b_side && fp32) { e.s_term_stride = (int64_t)(rows / 4) * (cols / blk) * 4; e.s_step = 0; }
-            else e.s_term_stride = 0;
+            // the four panels share one scale array (panel r is shifted by r * s_step rows / columns inside it)
+            e.s_term_stride = 0;
         } else {
             e.rows = (int)rows; e.cols = (int)cols; e.nq = 1; e.R = 1;
             e.coef[0][0] = 1.0f;
-            e.s_step = 0; e.s_ld = (int)cols; e.sf_blocks = (int)((b_side ? cols : rows) / 128);
+            e.s_step = 0; e.s_ld = (int)(b_side ? cols : rows); e.sf_blocks = (int)((b_side ? cols : rows) / 128);
         }
     } else {
         const float* cur = X;
@@ -176,7 +174,7 @@ fmm_status_t encode_side(const fmm_plan* plan, const FmmLayout& L, char* ws, con
         e.qoff[0] = 0; e.qoff[1] = e.cols; e.qoff[2] = (int64_t)e.rows * e.ld; e.qoff[3] = (int64_t)e.rows * e.ld + e.cols;
         for (int j = 0; j < 4; ++j) e.qoff_outer[j] = 2 * e.qoff[j];
         fill_coef(e.coef, coef, R);
-        e.s_step = 0; e.s_ld = e.cols; e.sf_blocks = (b_side ? e.cols : e.rows) / 128;
+        e.s_step = 0; e.s_ld = b_side ? e.cols : e.rows; e.sf_blocks = (b_side ? e.cols : e.rows) / 128;
         if (fused2) {
             s = b_side ? fmm_launch_encode2_b(e, mode, st) : fmm_launch_encode2_a(e, blk, mode, st);
             if (s == FMM_OK) ++*launches;
@@ -391,7 +389,8 @@ fmm_status_t fmm_quantized_view(const fmm_plan_t* plan, int64_t M, int64_t N, in
     const bool fp32 = plan->qp.scale_mode == FMM_SCALE_FP32_AMAX_DIV_448;
     if (side == 'A') {
         *q_offset = L.qa + (size_t)term * L.m * L.k; *q_rows = L.m; *q_cols = L.k;
-        *scale_offset = L.sa + (size_t)term * L.sa_term; *scale_rows = L.m; *scale_cols = nkb;
+        *scale_offset = L.sa + (size_t)term * L.sa_term;
+        if (fp32) { *scale_rows = L.k / 128; *scale_cols = L.m * (128 / plan->qp.block_k); } else { *scale_rows = L.m; *scale_cols = nkb; }
     } else {
         *q_offset = L.qb + (size_t)term * L.n * L.k; *q_rows = L.n; *q_cols = L.k;
         *scale_offset = L.sb + (size_t)term * L.sb_term;

@@ -164,7 +164,6 @@ __device__ __forceinline__ void store_chunk_a(const EncodeParams& p, const float
     constexpr int GROUP = BLK / 4;
     constexpr unsigned FULL = 0xffffffffu;
     const int64_t term_codes = (int64_t)p.rows * p.cols;
-    const int nkb = p.cols / BLK;
     const int my_r = lane & 7;
     uint8_t* qp = p.q_out + ((int64_t)b * p.R) * term_codes + (int64_t)i * p.cols + c * 128 + lane * 4;
 #pragma unroll
@@ -179,8 +178,12 @@ __device__ __forceinline__ void store_chunk_a(const EncodeParams& p, const float
     // scales: lane holds the scale of combination my_r, block (lane / GROUP) of this chunk
     if (MODE == FMM_SCALE_FP32_AMAX_DIV_448) {
         if (my_r < p.R && (GROUP == 8 || lane < 8)) {
+            // chunk-major: [128-k chunk c][row i][K block of the chunk], so the scales one pipeline stage of the
+            // product kernel needs for 128 rows are contiguous, and this warp's (up to four) scales are adjacent;
+            // combination my_r is shifted by my_r * s_step rows when several combinations share one array
+            // (row panels of a plain pass)
             float* so = reinterpret_cast<float*>(reinterpret_cast<char*>(p.s_out) + ((int64_t)b * p.R + my_r) * p.s_term_stride);
-            so[(int64_t)i * nkb + c * (128 / BLK) + (GROUP == 8 ? (lane >> 3) : 0)] = s;
+            so[((int64_t)c * p.s_ld + i + my_r * p.s_step) * (128 / BLK) + (GROUP == 8 ? (lane >> 3) : 0)] = s;
         }
     } else {
         // four exponent bytes of this row (blocks 4c .. 4c+3) form one aligned word of the scale tile

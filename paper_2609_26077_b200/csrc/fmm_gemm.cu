@@ -78,7 +78,11 @@ struct Cfg {
     static constexpr int SF_STAGE_BYTES = MX ? (512 + SFB_ATOMS * 512) : 0;
     static constexpr int KB_PER_STAGE = BK / BLK;
     static constexpr int SB_STAGES = STAGES + 1;
-    static constexpr int SB_STAGE_BYTES = MX ? 0 : KB_PER_STAGE * BN * 4;
+    // FP32 modes: one stage of the scale ring = the B-side scales of the stage's K blocks (KB x BN fp32, stored
+    // K-block-major) followed by the A-side scales of this CTA's 128 rows (128 x KB fp32: the A side stores the KB
+    // scales of a 128-k chunk next to each other per row, one contiguous piece per stage)
+    static constexpr int SB_PART_BYTES = MX ? 0 : KB_PER_STAGE * BN * 4;
+    static constexpr int SB_STAGE_BYTES = MX ? 0 : KB_PER_STAGE * (BN + BM) * 4;
     static constexpr int TX_BYTES = NCTA * (A_BYTES + B_BYTES + SF_STAGE_BYTES);
     static constexpr int TX_BYTES_HALF = NCTA * (A_BYTES + B_BYTES / 2 + 1024);   // half-width item: one SFB atom
     static constexpr int OFF_A = 0;
@@ -279,8 +283,10 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                 const int grp = slot / p.positions, pos = slot - grp * p.positions;
                 const int tn = pos % tiles_n;
                 const int t_end = (grp + 1) * p.terms_per_group;
+                const int tm = pos / tiles_n;
                 for (int t = t_end - p.terms_per_group; t < t_end && ok; ++t) {
                     const uint8_t* sb_t = p.sb + (long long)t * p.sb_term + (long long)tn * BN * 4;
+                    const uint8_t* sa_t = p.sa + (long long)t * p.sa_term + (long long)(tm * NCTA + cta_rank) * BM * (C::KB_PER_STAGE * 4);
                     for (int ks = 0; ks < kstages; ++ks) {
                         if (!mbar_wait(bar_sempty(ss), sphase ^ 1u, ctl, 102)) { ok = false; break; }
                         mbar_expect_tx(bar_sfull(ss), C::SB_STAGE_BYTES);
@@ -288,6 +294,8 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                         for (int g = 0; g < C::KB_PER_STAGE; ++g)
                             bulk_load(base + C::OFF_SB + ss * C::SB_STAGE_BYTES + g * BN * 4,
                                       sb_t + (long long)(ks * C::KB_PER_STAGE + g) * p.n * 4, BN * 4, bar_sfull(ss));
+                        bulk_load(base + C::OFF_SB + ss * C::SB_STAGE_BYTES + C::SB_PART_BYTES,
+                                  sa_t + (long long)ks * p.m * (C::KB_PER_STAGE * 4), BM * C::KB_PER_STAGE * 4, bar_sfull(ss));
                         if (++ss == C::SB_STAGES) { ss = 0; sphase ^= 1u; }
                     }
                 }
@@ -367,7 +375,9 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer (even CTA only in a pair)
-        if (lane == 0 && leader) {
+        // The whole warp walks the loops (convergent, warp-uniform operands); each tcgen05 instruction is issued by
+        // one elected lane inside its wrapper.
+        if (leader) {
             int stage = 0; uint32_t phase = 0;
             int buf = 0; uint32_t bphase = 0;
             bool ok = true;
@@ -381,11 +391,11 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                 const uint32_t idesc = half ? (idesc_full & ~(0x3Fu << 17)) | ((uint32_t)(BN >> 4) << 17) : idesc_full;
                 for (int t = 0; t < p.terms_per_group && ok; ++t) {
                     if (C::MX) {
-                        if (!mbar_wait(bar_tempty(0), bphase ^ 1u, ctl, 201)) { ok = false; break; }
+                        if (!mbar_wait_warp(bar_tempty(0), bphase ^ 1u, ctl, 201)) { ok = false; break; }
                         tc_fence_after();
                     }
                     for (int ks = 0; ks < kstages; ++ks) {
-                        if (!mbar_wait(bar_full(stage), phase, ctl, 202)) { ok = false; break; }
+                        if (!mbar_wait_warp(bar_full(stage), phase, ctl, 202)) { ok = false; break; }
                         tc_fence_after();
                         const uint64_t adesc = make_kmajor_sw128_desc(base + C::OFF_A + stage * C::A_BYTES);
                         const uint64_t bdesc = make_kmajor_sw128_desc(base + C::OFF_B + stage * C::B_BYTES);
@@ -405,7 +415,7 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                         } else {
 #pragma unroll
                             for (int g0 = 0; g0 < C::KB_PER_STAGE; g0 += C::GPB) {
-                                if (!mbar_wait(bar_tempty(buf), bphase ^ 1u, ctl, 203)) { ok = false; break; }
+                                if (!mbar_wait_warp(bar_tempty(buf), bphase ^ 1u, ctl, 203)) { ok = false; break; }
                                 tc_fence_after();
 #pragma unroll
                                 for (int gi = 0; gi < C::GPB; ++gi) {
@@ -480,25 +490,24 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                     for (int i = 0; i < C::CW / 2; ++i) acc2[i] = 0ull;         // acc2[k * (CW/8) + j]: row slot k, column group j
                     constexpr int JG = C::CW / 8;                               // column groups of eight per warp
                     constexpr int KB = C::KB_PER_STAGE;
-                    const float* sa_rows = reinterpret_cast<const float*>(p.sa + (long long)t * p.sa_term) +
-                                           (long long)(row_in_leaf + (lane >> 2)) * nkb;
-                    const int row_step = 8 * nkb;                               // eight rows further
+                    // A-side scales of the thread's four rows (q*32 + lane/4 + 8k of this CTA's 128), per K block
+                    const uint32_t sa_lane = base + C::OFF_SB + C::SB_PART_BYTES + (q * 32 + (lane >> 2)) * (KB * 4);
                     const uint32_t sb_lane = base + C::OFF_SB + (h * C::CW + 2 * (lane & 3)) * 4;
                     for (int ks = 0; ks < kstages && ok; ++ks) {
-                        // the four K blocks of this stage for the thread's four rows; issued before the waits below,
-                        // which cover the load latency (a second set in flight would cost 16 more registers)
+                        if (!mbar_wait_warp(bar_sfull(ss), sphase, ctl, 302)) { ok = false; break; }
+                        const uint32_t sbs32 = sb_lane + ss * C::SB_STAGE_BYTES;
+                        // the stage's K blocks for the thread's four rows, from the scale ring (a global load here, even
+                        // issued a stage early, stalled the promotion: 14 % of the block-32 kernel)
                         float sa4[4][KB];
 #pragma unroll
                         for (int k = 0; k < 4; ++k) {
                             if constexpr (KB == 4) {
-                                const float4 v4 = __ldg(reinterpret_cast<const float4*>(sa_rows + k * row_step) + ks);
+                                const float4 v4 = lds128(sa_lane + ss * C::SB_STAGE_BYTES + 8 * k * 16);
                                 sa4[k][0] = v4.x; sa4[k][1] = v4.y; sa4[k][2] = v4.z; sa4[k][3] = v4.w;
                             } else {
-                                sa4[k][0] = __ldg(sa_rows + (k * row_step + ks));
+                                sa4[k][0] = lds32f(sa_lane + ss * C::SB_STAGE_BYTES + 8 * k * 4);
                             }
                         }
-                        if (!mbar_wait_warp(bar_sfull(ss), sphase, ctl, 302)) { ok = false; break; }
-                        const uint32_t sbs32 = sb_lane + ss * C::SB_STAGE_BYTES;
 #pragma unroll
                         for (int g0 = 0; g0 < C::KB_PER_STAGE; g0 += C::GPB) {
                             if (!mbar_wait_warp(bar_tfull(buf), bphase, ctl, 303)) { ok = false; break; }
@@ -550,28 +559,13 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                 } else {
 #pragma unroll
                     for (int i = 0; i < C::CW / 2; ++i) acc2[i] = 0ull;
-                    const float* sa_row = reinterpret_cast<const float*>(p.sa + (long long)t * p.sa_term) +
-                                          (long long)(row_in_leaf + lane) * nkb;
-                    // row scales are prefetched PF stages ahead (each thread walks its own row of the scale matrix)
-                    constexpr int PF = (C::KB_PER_STAGE >= 4) ? 1 : 2;
-                    float sa_q[PF + 1][C::KB_PER_STAGE];
-#pragma unroll
-                    for (int d = 0; d < PF; ++d)
-#pragma unroll
-                        for (int g = 0; g < C::KB_PER_STAGE; ++g)
-                            sa_q[d][g] = (d < kstages) ? __ldg(sa_row + d * C::KB_PER_STAGE + g) : 0.0f;
+                    // this thread's row (q*32 + lane of the CTA's 128) in the A-side part of a scale stage
+                    const uint32_t sa_lane = base + C::OFF_SB + C::SB_PART_BYTES + (q * 32 + lane) * (C::KB_PER_STAGE * 4);
                     for (int ks = 0; ks < kstages && ok; ++ks) {
-#pragma unroll
-                        for (int g = 0; g < C::KB_PER_STAGE; ++g)
-                            sa_q[PF][g] = (ks + PF < kstages) ? __ldg(sa_row + (ks + PF) * C::KB_PER_STAGE + g) : 0.0f;
                         if (!mbar_wait_warp(bar_sfull(ss), sphase, ctl, 302)) { ok = false; break; }
                         float sa[C::KB_PER_STAGE];
 #pragma unroll
-                        for (int g = 0; g < C::KB_PER_STAGE; ++g) {
-                            sa[g] = sa_q[0][g];
-#pragma unroll
-                            for (int d = 0; d < PF; ++d) sa_q[d][g] = sa_q[d + 1][g];
-                        }
+                        for (int g = 0; g < C::KB_PER_STAGE; ++g) sa[g] = lds32f(sa_lane + ss * C::SB_STAGE_BYTES + g * 4);
                         const uint8_t* sbs = base_ptr + C::OFF_SB + ss * C::SB_STAGE_BYTES;
 #pragma unroll
                         for (int g0 = 0; g0 < C::KB_PER_STAGE; g0 += C::GPB) {

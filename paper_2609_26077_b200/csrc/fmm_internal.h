@@ -60,7 +60,7 @@ struct EncodeParams {
     void* s_out;              // scales
     int64_t s_term_stride;    // bytes between the scale arrays of consecutive terms
     int s_step;               // rows (A side) / columns (B side) by which combination r is shifted inside a shared scale array
-    int s_ld;                 // B side, fp32 scales: row length of the scale array
+    int s_ld;                 // fp32 scales: columns of B / rows of A that the shared scale array covers
     int sf_blocks;            // UE8M0: number of 128-row blocks of the scale-tile array
     float amax_floor;
     int b_tile;               // B side: 128 = one fp32 scale per 128 x 128 tile (blk 128 only), 0 = per column

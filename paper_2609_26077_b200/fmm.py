@@ -212,6 +212,10 @@ class Plan:
             scales = host[so:so + sr * sc * 4].view(np.float32).reshape(sr, sc)
             if side == "B":
                 codes = codes.T
+            else:
+                # stored [128-k chunk][row][K block of the chunk]
+                g = 128 // self.block_k
+                scales = scales.reshape(sr, sc // g, g).transpose(1, 0, 2).reshape(sc // g, sr * g)
         else:
             rows, nkb = sr, sc
             tiles = host[so:so + rows * nkb].reshape(nkb // 4, rows // 128, 32, 4, 4)   # [kb/4, r/128, r%32, (r%128)/32, kb%4]
