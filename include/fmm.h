@@ -191,6 +191,19 @@ int64_t fmm_error_stats_noalloc_max_elements(void);
  * call that set it are invalid.  Returns FMM_ERR_DEVICE_TIMEOUT when *code != 0. */
 fmm_status_t fmm_device_status(const fmm_plan_t* plan, int* code);
 
+/* Debug build (no counterpart in the paper).  The library can be built a second time with -DFMM_DEBUG
+ * (libfmm_b200_debug.so): every global store of every kernel is then checked against the buffers the launch was
+ * given (workspace slices, C, scratch); a store outside them is skipped and a location code is recorded - nothing
+ * traps and the context stays usable.  fmm_debug_build() tells which build is loaded (1 = debug).
+ * fmm_debug_violation synchronises the device and returns the first recorded code of the plan's launches (0 = none;
+ * plan == NULL: of the statistics / reference kernels, which take no plan).  In the normal build it always reports 0. */
+int fmm_debug_build(void);
+fmm_status_t fmm_debug_violation(const fmm_plan_t* plan, int* code);
+/* Self-test of that guard, safe in either build: enqueues a one-thread kernel that stores to a spare word of the
+ * plan's own status array under a guard that does not include that word.  Debug build: the store is skipped and
+ * fmm_debug_violation reports code 1901 until fmm_device_status_clear; normal build: no effect that a caller sees. */
+fmm_status_t fmm_selftest_store_guard(const fmm_plan_t* plan, void* cuda_stream);
+
 /* Resets the plan's status words to zero, after cudaDeviceSynchronize. */
 fmm_status_t fmm_device_status_clear(const fmm_plan_t* plan);
 

@@ -121,6 +121,8 @@ fmm_status_t encode_side(const fmm_plan* plan, const FmmLayout& L, char* ws, con
     e.amax_floor = plan->qp.amax_floor;
     e.b_tile = b_side ? plan->qp.b_tile_n : 0;
     e.preround_bf16 = (b_side && plan->qp.b_preround_bf16) ? 1 : 0;
+    e.guard = fmm_make_guard(e.q_out, (size_t)L.terms * (size_t)((b_side ? L.n : L.m) * L.k),
+                             e.s_out, (size_t)L.terms * (b_side ? L.sb_term : L.sa_term), plan->d_status + FMM_GUARD_WORD);
     fmm_status_t s;
     if (lv == 0) {
         // Plain quantization of the matrix itself.  The matrix is cut into four panels (row panels of A,
@@ -162,6 +164,8 @@ fmm_status_t encode_side(const fmm_plan* plan, const FmmLayout& L, char* ws, con
             c.rows = (int)(cur_rows / 2); c.cols = (int)(cur_cols / 2); c.R = R;
             fill_coef(c.coef, coef, R);
             c.out = reinterpret_cast<float*>(ws + (b_side ? L.inter_b[level] : L.inter_a[level]));
+            c.guard = fmm_make_guard(c.out, (size_t)batch * R * (size_t)(c.rows * (int64_t)c.cols) * 4, nullptr, 0,
+                                     plan->d_status + FMM_GUARD_WORD);
             s = fmm_launch_comb(c, st);
             if (s != FMM_OK) return s;
             ++*launches;
@@ -209,6 +213,7 @@ fmm_status_t multiply(const fmm_plan* plan, const FmmLayout& L, char* ws, float*
     g.terms_per_group = plan->levels >= 2 ? plan->rank : (int)L.terms;
     g.out_start = plan->d_out_start; g.out = plan->d_out; g.status = plan->d_status;
     g.sb_tile = plan->qp.b_tile_n == 128 ? 1 : 0;
+    g.guard = fmm_make_guard(dest, (size_t)g.Mfull * (size_t)g.Nfull * 4, nullptr, 0, plan->d_status + FMM_GUARD_WORD);
     fmm_status_t s = fmm_launch_gemm(g, plan->qp.block_k, (int)plan->qp.scale_mode, st, launches);
     if (s != FMM_OK) return s;
     for (int l = lv - 1; l >= 1; --l) {
@@ -220,6 +225,8 @@ fmm_status_t multiply(const fmm_plan* plan, const FmmLayout& L, char* ws, float*
         d.rows = (int)(M >> l); d.cols = (int)(N >> l); d.R = plan->rank;
         for (int r = 0; r < plan->rank; ++r)
             for (int q = 0; q < 4; ++q) d.W[r][q] = plan->W[r][q];
+        d.guard = fmm_make_guard(d.out, (size_t)d.batch * 4 * (size_t)d.rows * (size_t)d.cols * 4, nullptr, 0,
+                                 plan->d_status + FMM_GUARD_WORD);
         s = fmm_launch_decode(d, st);
         if (s != FMM_OK) return s;
         ++*launches;
@@ -497,6 +504,26 @@ fmm_status_t fmm_device_status(const fmm_plan_t* plan, int* code)
     return h[0] ? FMM_ERR_DEVICE_TIMEOUT : FMM_OK;
 }
 
+int fmm_debug_build(void)
+{
+#ifdef FMM_DEBUG
+    return 1;
+#else
+    return 0;
+#endif
+}
+
+fmm_status_t fmm_debug_violation(const fmm_plan_t* plan, int* code)
+{
+    if (!code) return FMM_ERR_INVALID_ARG;
+    if (!plan) return fmm_stats_guard_read(code);
+    fmm_status_t sd = check_device(plan);
+    if (sd != FMM_OK) return sd;
+    if (cudaDeviceSynchronize() != cudaSuccess) { cudaGetLastError(); return FMM_ERR_CUDA; }
+    if (cudaMemcpy(code, plan->d_status + FMM_GUARD_WORD, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) { cudaGetLastError(); return FMM_ERR_CUDA; }
+    return FMM_OK;
+}
+
 fmm_status_t fmm_device_status_clear(const fmm_plan_t* plan)
 {
     if (!plan) return FMM_ERR_INVALID_ARG;
@@ -513,6 +540,14 @@ fmm_status_t fmm_selftest_bounded_wait(const fmm_plan_t* plan, int64_t limit_ns,
     fmm_status_t sd = check_device(plan);
     if (sd != FMM_OK) return sd;
     return fmm_launch_bounded_wait_selftest(plan->d_status, (unsigned long long)limit_ns, reinterpret_cast<cudaStream_t>(stream));
+}
+
+fmm_status_t fmm_selftest_store_guard(const fmm_plan_t* plan, void* stream)
+{
+    if (!plan) return FMM_ERR_INVALID_ARG;
+    fmm_status_t sd = check_device(plan);
+    if (sd != FMM_OK) return sd;
+    return fmm_launch_guard_selftest(plan->d_status, reinterpret_cast<cudaStream_t>(stream));
 }
 
 fmm_status_t fmm_last_launch_count(const fmm_plan_t* plan, int* launches)

@@ -170,6 +170,7 @@ __device__ __forceinline__ void store_chunk_a(const EncodeParams& p, const float
     for (int r = 0; r < FMM_MAX_RANK; ++r) {
         if (row_used<NZ>(r, p.R)) {
             const float inv_r = __shfl_sync(FULL, inv, (GROUP == 32) ? r : ((lane & 24) | r));
+            if (FMM_GUARD(p.guard, qp, 4, 1101))
             *reinterpret_cast<uint32_t*>(qp) = pack4_e4m3(__fmul_rn(v[r].x, inv_r), __fmul_rn(v[r].y, inv_r),
                                                           __fmul_rn(v[r].z, inv_r), __fmul_rn(v[r].w, inv_r));
         }
@@ -183,7 +184,8 @@ __device__ __forceinline__ void store_chunk_a(const EncodeParams& p, const float
             // combination my_r is shifted by my_r * s_step rows when several combinations share one array
             // (row panels of a plain pass)
             float* so = reinterpret_cast<float*>(reinterpret_cast<char*>(p.s_out) + ((int64_t)b * p.R + my_r) * p.s_term_stride);
-            so[((int64_t)c * p.s_ld + i + my_r * p.s_step) * (128 / BLK) + (GROUP == 8 ? (lane >> 3) : 0)] = s;
+            float* sp = so + ((int64_t)c * p.s_ld + i + my_r * p.s_step) * (128 / BLK) + (GROUP == 8 ? (lane >> 3) : 0);
+            if (FMM_GUARD(p.guard, sp, 4, 1102)) *sp = s;
         }
     } else {
         // four exponent bytes of this row (blocks 4c .. 4c+3) form one aligned word of the scale tile
@@ -194,7 +196,8 @@ __device__ __forceinline__ void store_chunk_a(const EncodeParams& p, const float
             char* so = reinterpret_cast<char*>(p.s_out) + ((int64_t)b * p.R + lane) * p.s_term_stride;
             const int ig = i + lane * p.s_step;            // row inside the scale-tile array
             const int64_t tile = (int64_t)c * p.sf_blocks + (ig >> 7);
-            *reinterpret_cast<uint32_t*>(so + tile * 512 + (ig & 31) * 16 + ((ig & 127) >> 5) * 4) = wv;
+            char* sp = so + tile * 512 + (ig & 31) * 16 + ((ig & 127) >> 5) * 4;
+            if (FMM_GUARD(p.guard, sp, 4, 1103)) *reinterpret_cast<uint32_t*>(sp) = wv;
         }
     }
 }
@@ -264,10 +267,12 @@ __device__ __forceinline__ void store_b_scale(const EncodeParams& p, int64_t t, 
     char* so = reinterpret_cast<char*>(p.s_out) + t * p.s_term_stride;
     const int jg = j + r * p.s_step;                   // column inside the scale array
     if (MODE == FMM_SCALE_FP32_AMAX_DIV_448) {
-        reinterpret_cast<float*>(so)[(int64_t)kb * p.s_ld + jg] = s;
+        float* sp = reinterpret_cast<float*>(so) + (int64_t)kb * p.s_ld + jg;
+        if (FMM_GUARD(p.guard, sp, 4, 1201)) *sp = s;
     } else if (last_of_word) {
         const int64_t tile = (int64_t)kc * p.sf_blocks + (jg >> 7);
-        *reinterpret_cast<uint32_t*>(so + tile * 512 + (jg & 31) * 16 + ((jg & 127) >> 5) * 4) = e8word;
+        char* sp = so + tile * 512 + (jg & 31) * 16 + ((jg & 127) >> 5) * 4;
+        if (FMM_GUARD(p.guard, sp, 4, 1202)) *reinterpret_cast<uint32_t*>(sp) = e8word;
     }
 }
 
@@ -355,8 +360,8 @@ __global__ void __launch_bounds__(TILE ? 256 : 128, TILE ? 2 : 4) encode_b_kerne
                         for (int g = 0; g < 4; ++g)
                             wv[g] = pack4_e4m3(__fmul_rn(v[4 * g], inv), __fmul_rn(v[4 * g + 1], inv),
                                                __fmul_rn(v[4 * g + 2], inv), __fmul_rn(v[4 * g + 3], inv));
-                        *reinterpret_cast<uint4*>(p.q_out + t * term_codes + (int64_t)j * p.rows + k0) =
-                            make_uint4(wv[0], wv[1], wv[2], wv[3]);
+                        uint8_t* qp = p.q_out + t * term_codes + (int64_t)j * p.rows + k0;
+                        if (FMM_GUARD(p.guard, qp, 16, 1203)) *reinterpret_cast<uint4*>(qp) = make_uint4(wv[0], wv[1], wv[2], wv[3]);
                     }
                 }
             }
@@ -489,6 +494,7 @@ __global__ void __launch_bounds__(256) encode2_b_kernel(const EncodeParams p)
             for (int r = 0; r < FMM_MAX_RANK; ++r) {
                 if (row_used<NZ>(r, p.R)) {
                     const float inv_r = __shfl_sync(FULL, inv, (lane & 24) | r);
+                    if (FMM_GUARD(p.guard, qp, 4, 1301))
                     *reinterpret_cast<uint32_t*>(qp) = pack4_e4m3(__fmul_rn(v[r].x, inv_r), __fmul_rn(v[r].y, inv_r),
                                                                   __fmul_rn(v[r].z, inv_r), __fmul_rn(v[r].w, inv_r));
                 }
@@ -497,10 +503,12 @@ __global__ void __launch_bounds__(256) encode2_b_kernel(const EncodeParams p)
             if (my_r < p.R) {
                 char* so = reinterpret_cast<char*>(p.s_out) + (t0 + my_r) * p.s_term_stride;
                 if (MODE == FMM_SCALE_FP32_AMAX_DIV_448) {
-                    reinterpret_cast<float*>(so)[(int64_t)kb * p.s_ld + j] = s;
+                    float* sp = reinterpret_cast<float*>(so) + (int64_t)kb * p.s_ld + j;
+                    if (FMM_GUARD(p.guard, sp, 4, 1302)) *sp = s;
                 } else {
                     const int64_t tile = (int64_t)(kb >> 2) * p.sf_blocks + (j >> 7);
-                    *reinterpret_cast<uint8_t*>(so + tile * 512 + (j & 31) * 16 + ((j & 127) >> 5) * 4 + (kb & 3)) = (uint8_t)e8;
+                    char* sp = so + tile * 512 + (j & 31) * 16 + ((j & 127) >> 5) * 4 + (kb & 3);
+                    if (FMM_GUARD(p.guard, sp, 1, 1303)) *reinterpret_cast<uint8_t*>(sp) = (uint8_t)e8;
                 }
             }
         }
@@ -540,7 +548,7 @@ __global__ void __launch_bounds__(256) comb_kernel(const CombParams p)
                 }
             }
             float* o = p.out + ((int64_t)b * p.R + r) * p.rows * p.cols + (int64_t)i * p.cols + c * 4;
-            *reinterpret_cast<float4*>(o) = v;
+            if (FMM_GUARD(p.guard, o, 16, 1401)) *reinterpret_cast<float4*>(o) = v;
         }
     }
 }
@@ -590,8 +598,10 @@ __global__ void __launch_bounds__(256) decode_kernel(const DecodeParams p)
         }
         float* dst = p.out + (int64_t)b * 4 * in_stride;
 #pragma unroll
-        for (int q = 0; q < 4; ++q)
-            *reinterpret_cast<float4*>(dst + ((int64_t)(q >> 1) * p.rows + i) * out_ld + (q & 1) * p.cols + c * 4) = acc[q];
+        for (int q = 0; q < 4; ++q) {
+            float* o = dst + ((int64_t)(q >> 1) * p.rows + i) * out_ld + (q & 1) * p.cols + c * 4;
+            if (FMM_GUARD(p.guard, o, 16, 1501)) *reinterpret_cast<float4*>(o) = acc[q];
+        }
     }
 }
 

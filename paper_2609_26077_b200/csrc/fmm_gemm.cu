@@ -169,6 +169,8 @@ struct KParams {
     int positions, terms_per_group, split_from, items;
     const int* out_start; const FmmOutEntry* out;
     int* status;
+    const float* c_base; long long ldc;       // the output matrix as plain memory: used by the FMM_DEBUG store guard only
+    FmmGuard guard;
 };
 
 template <int BN, int MODE, int BLK, int NCTA>
@@ -358,6 +360,7 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                                 for (int k = 0; k < C::OUT_BUFS / 2; ++k) {
                                     const int ch = ch0 + k;
                                     const int r = row0 + (ch / (BN / 32)) * 32, c = col0 + (ch % (BN / 32)) * 32;
+                                    if (!FMM_GUARD(p.guard, p.c_base + (long long)r * p.ldc + c, (31 * p.ldc + 32) * 4, 1701)) continue;
                                     if (ent.first) tma_store_2d_hint(&tmC, c, r, stg + (b0 + k) * 4096, pol_c);      // lane 0: stg = chunk base
                                     else tma_reduce_add_2d_hint(&tmC, c, r, stg + (b0 + k) * 4096, pol_c);
                                 }
@@ -683,8 +686,10 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                         fence_proxy_async();
                         __syncwarp();
                         if (lane == 0) {
-                            if (ent.first) tma_store_2d_hint(&tmC, col0 + c * C::CH, row0, stg + b * C::STAGING_BYTES, pol_c);
-                            else tma_reduce_add_2d_hint(&tmC, col0 + c * C::CH, row0, stg + b * C::STAGING_BYTES, pol_c);
+                            if (FMM_GUARD(p.guard, p.c_base + (long long)row0 * p.ldc + col0 + c * C::CH, (31 * p.ldc + C::CH) * 4, 1702)) {
+                                if (ent.first) tma_store_2d_hint(&tmC, col0 + c * C::CH, row0, stg + b * C::STAGING_BYTES, pol_c);
+                                else tma_reduce_add_2d_hint(&tmC, col0 + c * C::CH, row0, stg + b * C::STAGING_BYTES, pol_c);
+                            }
                             bulk_commit();
                         }
                         ++store_cnt;
@@ -802,6 +807,7 @@ fmm_status_t launch(const GemmParams& g, cudaStream_t st)
     kp.split_from = split ? slots - tail : slots;
     kp.items = slots + (split ? tail : 0);
     kp.out_start = g.out_start; kp.out = g.out; kp.status = g.status;
+    kp.c_base = g.C; kp.ldc = g.Nfull; kp.guard = g.guard;
 
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof(cfg));

@@ -18,6 +18,38 @@ struct FmmOutEntry {
     int first;     // 1: overwrite, 0: add
 };
 
+// Store guard of the FMM_DEBUG build (the stand-in for a memory checker, which this library cannot count on
+// having): the address ranges a launch may write, and where to report a store that falls outside them.  Every
+// launch fills it in; the kernels test it only when compiled with -DFMM_DEBUG - a bad store is then skipped and its
+// location code goes to *status (first one wins, nothing traps).
+struct FmmGuard {
+    const char* lo[2];
+    const char* hi[2];
+    int* status;
+};
+#if defined(FMM_DEBUG) && defined(__CUDACC__)
+__device__ __forceinline__ bool fmm_guard_ok(const FmmGuard& g, const void* ptr, size_t bytes, int code)
+{
+    const char* c = static_cast<const char*>(ptr);
+    if ((c >= g.lo[0] && c + bytes <= g.hi[0]) || (c >= g.lo[1] && c + bytes <= g.hi[1])) return true;
+    if (g.status) atomicCAS(g.status, 0, code);
+    return false;
+}
+#define FMM_GUARD(g, ptr, bytes, code) fmm_guard_ok(g, ptr, bytes, code)
+#else
+#define FMM_GUARD(g, ptr, bytes, code) true
+#endif
+static inline FmmGuard fmm_make_guard(const void* a, size_t na, const void* b, size_t nb, int* status)
+{
+    FmmGuard g;
+    g.lo[0] = static_cast<const char*>(a); g.hi[0] = g.lo[0] + na;
+    g.lo[1] = static_cast<const char*>(b); g.hi[1] = g.lo[1] + nb;
+    g.status = status;
+    return g;
+}
+// status word that receives guard violations: plan->d_status[FMM_GUARD_WORD]
+#define FMM_GUARD_WORD 2
+
 struct FmmLayout {            // byte offsets into the workspace
     int64_t m, n, k;          // leaf dimensions
     int64_t terms;            // R^levels (1 for levels == 0)
@@ -65,6 +97,7 @@ struct EncodeParams {
     float amax_floor;
     int b_tile;               // B side: 128 = one fp32 scale per 128 x 128 tile (blk 128 only), 0 = per column
     int preround_bf16;        // B side: round each combination to bfloat16 before the maximum and the cast
+    FmmGuard guard;           // codes and scales of this side
 };
 
 struct CombParams {
@@ -73,6 +106,7 @@ struct CombParams {
     int batch, rows, cols, R;
     float coef[FMM_MAX_RANK][4];
     float* out;               // dense rows x cols per (b, r)
+    FmmGuard guard;
 };
 
 // One outward step of the decoder: out[b] (2*rows x 2*cols, block q at (q>>1, q&1)) = sum_r W[r][q] * in[b*R + r]
@@ -81,6 +115,7 @@ struct DecodeParams {
     float* out;               // batch matrices, 2*rows x 2*cols each, dense
     int batch, rows, cols, R;
     float W[FMM_MAX_RANK][4];
+    FmmGuard guard;
 };
 fmm_status_t fmm_launch_decode(const DecodeParams& p, cudaStream_t st);
 fmm_status_t fmm_launch_comb(const CombParams& p, cudaStream_t st);
@@ -102,8 +137,12 @@ struct GemmParams {
     int* status;
     int terms_per_group;                    // consecutive terms that feed the same output blocks (R at levels >= 2, else all)
     int sb_tile;                            // fp32 scales, blk 128: the B-side scale is constant over each 128-column tile
+    FmmGuard guard;                         // the output matrix (C, or the stack of parent matrices)
 };
+// guard word of the statistics kernels, which have no plan (FMM_DEBUG build; always 0 otherwise)
+fmm_status_t fmm_stats_guard_read(int* code);
 fmm_status_t fmm_launch_bounded_wait_selftest(int* status, unsigned long long limit_ns, cudaStream_t st);
+fmm_status_t fmm_launch_guard_selftest(int* status, cudaStream_t st);
 fmm_status_t fmm_launch_gemm(const GemmParams& p, int blk, int mode, cudaStream_t st, int* launches);
 
 static inline int64_t fmm_ipow(int64_t b, int e) { int64_t r = 1; while (e-- > 0) r *= b; return r; }

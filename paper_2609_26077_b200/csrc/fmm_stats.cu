@@ -12,6 +12,8 @@
 // In host code this name is only a stand-in for the symbol; the device address comes from
 // cudaGetSymbolAddress (see noalloc_scratch below).
 static __device__ __align__(256) double g_noalloc_partials[3 * 1024];
+// where the statistics kernels of the FMM_DEBUG build report a store outside their output buffers
+static __device__ int g_stats_guard_code;
 
 namespace {
 
@@ -47,7 +49,8 @@ __device__ __forceinline__ void block_reduce3(double& a, double& b, double& c, d
 
 __global__ void __launch_bounds__(STAT_THREADS) error_partial_kernel(const float* __restrict__ C,
                                                                     const double* __restrict__ Cref,
-                                                                    int64_t count, double* __restrict__ partial)
+                                                                    int64_t count, double* __restrict__ partial,
+                                                                    const FmmGuard guard)
 {
     __shared__ double sm[3 * (STAT_THREADS / 32)];
     double sd = 0.0, sr = 0.0, mx = 0.0;
@@ -73,13 +76,13 @@ __global__ void __launch_bounds__(STAT_THREADS) error_partial_kernel(const float
     }
     for (; i < pairs; i += stride) add(__ldcs(C2 + i), __ldcs(R2 + i));
     block_reduce3(sd, sr, mx, sm);
-    if (threadIdx.x == 0) {
+    if (threadIdx.x == 0 && FMM_GUARD(guard, partial + blockIdx.x * 3, 24, 1601)) {
         partial[blockIdx.x * 3] = sd; partial[blockIdx.x * 3 + 1] = sr; partial[blockIdx.x * 3 + 2] = mx;
     }
 }
 
 __global__ void __launch_bounds__(STAT_THREADS) error_final_kernel(const double* __restrict__ partial, int n,
-                                                                  double* __restrict__ out3)
+                                                                  double* __restrict__ out3, const FmmGuard guard)
 {
     __shared__ double sm[3 * (STAT_THREADS / 32)];
     double sd = 0.0, sr = 0.0, mx = 0.0;
@@ -87,12 +90,13 @@ __global__ void __launch_bounds__(STAT_THREADS) error_final_kernel(const double*
         sd += partial[i * 3]; sr += partial[i * 3 + 1]; mx = fmax(mx, partial[i * 3 + 2]);
     }
     block_reduce3(sd, sr, mx, sm);
-    if (threadIdx.x == 0) { out3[0] = sd; out3[1] = sr; out3[2] = mx; }
+    if (threadIdx.x == 0 && FMM_GUARD(guard, out3, 24, 1602)) { out3[0] = sd; out3[1] = sr; out3[2] = mx; }
 }
 
 // 64x64 output tile per block of 16x16 threads, 4x4 outputs per thread, K step 16.
 __global__ void __launch_bounds__(256) ref_gemm_fp64_kernel(const float* __restrict__ A, const float* __restrict__ B,
-                                                           double* __restrict__ C, int64_t M, int64_t N, int64_t K)
+                                                           double* __restrict__ C, int64_t M, int64_t N, int64_t K,
+                                                           const FmmGuard guard)
 {
     __shared__ float As[16][64 + 1];   // [k][m]
     __shared__ float Bs[16][64];       // [k][n]
@@ -135,12 +139,52 @@ __global__ void __launch_bounds__(256) ref_gemm_fp64_kernel(const float* __restr
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
         double* c = C + (m0 + ty * 4 + i) * N + n0 + tx * 4;
+        if (!FMM_GUARD(guard, c, 32, 1603)) continue;
         reinterpret_cast<double2*>(c)[0] = make_double2(acc[i][0], acc[i][1]);
         reinterpret_cast<double2*>(c)[1] = make_double2(acc[i][2], acc[i][3]);
     }
 }
 
+// Device address of g_stats_guard_code on the current device (FMM_DEBUG build; the release build passes no word and
+// never resolves the symbol, so its calls stay free of runtime lookups).
+int* stats_guard_word()
+{
+#ifdef FMM_DEBUG
+    int* ptr = nullptr;
+    if (cudaGetSymbolAddress((void**)&ptr, g_stats_guard_code) != cudaSuccess) { cudaGetLastError(); return nullptr; }
+    return ptr;
+#else
+    return nullptr;
+#endif
+}
+
 }  // namespace
+
+// Self-test of the store guard: one thread stores to status word 40 under a guard that allows words 32..39 only.
+// Both addresses lie inside the plan's 64-word status array, so nothing is ever written out of bounds; the checked
+// build must skip the store and record code 1901, the normal build has no guard and simply writes the spare word.
+__global__ void guard_selftest_kernel(int* status, const FmmGuard guard)
+{
+    int* target = status + 40;
+    if (FMM_GUARD(guard, target, sizeof(int), 1901)) *target = 1;
+}
+
+fmm_status_t fmm_launch_guard_selftest(int* status, cudaStream_t st)
+{
+    const FmmGuard guard = fmm_make_guard(status + 32, 8 * sizeof(int), nullptr, 0, status + FMM_GUARD_WORD);
+    guard_selftest_kernel<<<1, 1, 0, st>>>(status, guard);
+    return cudaGetLastError() == cudaSuccess ? FMM_OK : FMM_ERR_CUDA;
+}
+
+fmm_status_t fmm_stats_guard_read(int* code)
+{
+    *code = 0;
+#ifdef FMM_DEBUG
+    if (cudaDeviceSynchronize() != cudaSuccess) { cudaGetLastError(); return FMM_ERR_CUDA; }
+    if (cudaMemcpyFromSymbol(code, g_stats_guard_code, sizeof(int)) != cudaSuccess) { cudaGetLastError(); return FMM_ERR_CUDA; }
+#endif
+    return FMM_OK;
+}
 
 extern "C" {
 
@@ -156,8 +200,9 @@ fmm_status_t fmm_error_stats(const float* C, const double* Cref, int64_t M, int6
     if (((uintptr_t)C & 7) || ((uintptr_t)Cref & 15)) return FMM_ERR_INVALID_ARG;
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
     double* partial = static_cast<double*>(scratch);
-    error_partial_kernel<<<STAT_BLOCKS, STAT_THREADS, 0, st>>>(C, Cref, M * N, partial);
-    error_final_kernel<<<1, STAT_THREADS, 0, st>>>(partial, STAT_BLOCKS, out3);
+    const FmmGuard guard = fmm_make_guard(partial, sizeof(double) * 3 * STAT_BLOCKS, out3, sizeof(double) * 3, stats_guard_word());
+    error_partial_kernel<<<STAT_BLOCKS, STAT_THREADS, 0, st>>>(C, Cref, M * N, partial, guard);
+    error_final_kernel<<<1, STAT_THREADS, 0, st>>>(partial, STAT_BLOCKS, out3, guard);
     return cudaGetLastError() == cudaSuccess ? FMM_OK : FMM_ERR_CUDA;
 }
 
@@ -168,7 +213,8 @@ fmm_status_t fmm_ref_gemm_fp64(const float* A, const float* B, double* Cref, int
     if (M <= 0 || N <= 0 || K <= 0 || (M % 64) || (N % 64) || (K % 16)) return FMM_ERR_SHAPE;
     if ((uintptr_t)Cref & 15) return FMM_ERR_INVALID_ARG;
     dim3 grid((unsigned)(N / 64), (unsigned)(M / 64));
-    ref_gemm_fp64_kernel<<<grid, 256, 0, reinterpret_cast<cudaStream_t>(stream)>>>(A, B, Cref, M, N, K);
+    const FmmGuard guard = fmm_make_guard(Cref, sizeof(double) * (size_t)M * (size_t)N, nullptr, 0, stats_guard_word());
+    ref_gemm_fp64_kernel<<<grid, 256, 0, reinterpret_cast<cudaStream_t>(stream)>>>(A, B, Cref, M, N, K, guard);
     return cudaGetLastError() == cudaSuccess ? FMM_OK : FMM_ERR_CUDA;
 }
 
@@ -212,8 +258,9 @@ fmm_status_t fmm_error_stats_noalloc(const float* C, const double* Cref, int64_t
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
     // every one of the STAT_BLOCKS slots is rewritten by the first kernel, so nothing left behind by
     // an earlier call is ever read and no clearing is needed
-    error_partial_kernel<<<STAT_BLOCKS, STAT_THREADS, 0, st>>>(C, Cref, M * N, partial);
-    error_final_kernel<<<1, STAT_THREADS, 0, st>>>(partial, STAT_BLOCKS, out3);
+    const FmmGuard guard = fmm_make_guard(partial, sizeof(double) * 3 * STAT_BLOCKS, out3, sizeof(double) * 3, stats_guard_word());
+    error_partial_kernel<<<STAT_BLOCKS, STAT_THREADS, 0, st>>>(C, Cref, M * N, partial, guard);
+    error_final_kernel<<<1, STAT_THREADS, 0, st>>>(partial, STAT_BLOCKS, out3, guard);
     return cudaGetLastError() == cudaSuccess ? FMM_OK : FMM_ERR_CUDA;
 }
 

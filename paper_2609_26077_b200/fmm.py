@@ -8,7 +8,9 @@ import os
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libfmm_b200.so")
+# FMM_B200_DEBUG=1 in the environment selects the checked build (-DFMM_DEBUG: every global store of every kernel is
+# range-checked, see fmm_debug_violation); it is slower and meant for tests
+LIB_PATH = os.path.join(_HERE, "libfmm_b200_debug.so" if os.environ.get("FMM_B200_DEBUG") == "1" else "libfmm_b200.so")
 
 FMM_OK = 0
 STATUS_NAMES = ["FMM_OK", "FMM_ERR_INVALID_ARG", "FMM_ERR_SHAPE", "FMM_ERR_NOT_EXACT", "FMM_ERR_WORKSPACE",
@@ -21,7 +23,8 @@ EXPORTS = ["fmm_plan_create", "fmm_plan_destroy", "fmm_workspace_bytes", "fmm_ma
            "fmm_multiply_only", "fmm_quantized_view", "fmm_ref_gemm_fp64", "fmm_error_stats",
            "fmm_error_stats_scratch_bytes", "fmm_error_stats_noalloc", "fmm_error_stats_noalloc_max_elements",
            "fmm_device_status", "fmm_device_status_clear", "fmm_selftest_bounded_wait", "fmm_phi_gamma", "fmm_brent_residual",
-           "fmm_last_launch_count", "fmm_status_string"]
+           "fmm_last_launch_count", "fmm_status_string", "fmm_debug_build", "fmm_debug_violation",
+           "fmm_selftest_store_guard"]
 
 
 class QuantParams(C.Structure):
@@ -51,6 +54,7 @@ def lib():
         L.fmm_status_string.argtypes = [C.c_int]
         L.fmm_error_stats_scratch_bytes.restype = C.c_size_t
         L.fmm_error_stats_noalloc_max_elements.restype = C.c_int64
+        L.fmm_debug_build.restype = C.c_int
         for name in EXPORTS:
             getattr(L, name)
         _lib = L
