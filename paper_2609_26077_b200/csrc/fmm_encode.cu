@@ -211,31 +211,39 @@ __global__ void __launch_bounds__(256) encode_a_kernel(const EncodeParams p)
     const uint32_t warp_gid = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const uint32_t nwarps = (gridDim.x * blockDim.x) >> 5;
     const int chunks = p.cols / 128;
-    // a task is CPT consecutive 128-k chunks of one output row; tasks are dealt to warps round-robin
-    // (32-bit index arithmetic only: one division per task, none per chunk)
+    // a task is CPT consecutive 128-k chunks of one output row - with fp32 scales of TWO adjacent rows, walked chunk by
+    // chunk with the two rows of a chunk back to back: the fp32 scales of a chunk are stored row after row (16 bytes
+    // per row and chunk), so the two rows complete a 32-byte sector within two consecutive stores of this warp.  Tasks are dealt to warps
+    // round-robin (32-bit index arithmetic only: one division per task, none per chunk).
     const int CPT = (chunks % 8 == 0) ? 8 : ((chunks % 4 == 0) ? 4 : 1);
+    // (the power-of-two mode writes its exponent bytes in row-major tiles and is faster one row at a time)
+    const int RPT = (MODE == FMM_SCALE_FP32_AMAX_DIV_448 && p.rows % 2 == 0) ? 2 : 1;
     const uint32_t tasks_per_row = (uint32_t)(chunks / CPT);
-    const uint32_t tasks = (uint32_t)p.batch * (uint32_t)p.rows * tasks_per_row;
+    const uint32_t row_groups = (uint32_t)(p.rows / RPT);
+    const uint32_t tasks = (uint32_t)p.batch * row_groups * tasks_per_row;
 
     for (uint32_t task = warp_gid; task < tasks; task += nwarps) {
       const uint32_t row_id = task / tasks_per_row;
       const int c0 = (int)(task - row_id * tasks_per_row) * CPT;
-      const int b = (int)(row_id / (uint32_t)p.rows);
-      const int i = (int)(row_id - (uint32_t)b * (uint32_t)p.rows);
-      // the loads of chunk c+1 are issued before chunk c is processed (two chunks in flight per warp)
-      const float* row_base = p.in + (int64_t)b * p.in_batch_stride + (int64_t)i * p.ld + lane * 4;
+      const int b = (int)(row_id / row_groups);
+      const int i0 = (int)(row_id - (uint32_t)b * row_groups) * RPT;
+      // the loads of step n+1 are issued before step n is processed (two steps in flight per warp); step = (chunk, row)
+      const float* row_base = p.in + (int64_t)b * p.in_batch_stride + (int64_t)i0 * p.ld + lane * 4;
+      const int steps = CPT * RPT;
       float4 xn[4];
 #pragma unroll
       for (int j = 0; j < 4; ++j)
           if (j < p.nq) xn[j] = __ldcs(reinterpret_cast<const float4*>(row_base + c0 * 128 + p.qoff[j]));
-      for (int c = c0; c < c0 + CPT; ++c) {
+      for (int st = 0; st < steps; ++st) {
+        const int c = c0 + st / RPT, i = i0 + st % RPT;
         float4 x[4];
 #pragma unroll
         for (int j = 0; j < 4; ++j) x[j] = xn[j];
-        if (c + 1 < c0 + CPT) {
+        if (st + 1 < steps) {
+            const int cn = c0 + (st + 1) / RPT, rn = (st + 1) % RPT;
 #pragma unroll
             for (int j = 0; j < 4; ++j)
-                if (j < p.nq) xn[j] = __ldcs(reinterpret_cast<const float4*>(row_base + (c + 1) * 128 + p.qoff[j]));
+                if (j < p.nq) xn[j] = __ldcs(reinterpret_cast<const float4*>(row_base + (int64_t)rn * p.ld + cn * 128 + p.qoff[j]));
         }
 
         float4 v[FMM_MAX_RANK];
@@ -387,6 +395,89 @@ __global__ void __launch_bounds__(TILE ? 256 : 128, TILE ? 2 : 4) encode_b_kerne
                     if (khalf == 0) store_b_scale<MODE>(p, (int64_t)b * p.R + r, r, j, kc, kc, sc, 0u, false);
                 }
             }
+        }
+    }
+}
+
+// B side, block 128, per-column scales, one pass.  The four warps of a block take the four 32-k sub-blocks of one
+// 128-k block of the same 16 columns; every thread forms the combinations of its 16 k x 1 column, the sub-block
+// maxima meet in shared memory, and each warp then quantizes its own sub-block from the raw values it still holds
+// (the combinations are formed a second time in registers - the same rounded-multiply / FMA chain, so the same bits -
+// instead of reading the operand a second time).  Grid: (cols / 16, rows / 128, batch), 128 threads.
+template <uint32_t NZ>
+__global__ void __launch_bounds__(128, 4) encode_b128_kernel(const EncodeParams p)
+{
+    constexpr unsigned FULL = 0xffffffffu;
+    constexpr int MODE = FMM_SCALE_FP32_AMAX_DIV_448;
+    __shared__ float sub_amax[4][FMM_MAX_RANK][16];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int col = lane & 15, khalf = lane >> 4;
+    const int j = blockIdx.x * 16 + col;
+    const int kc = blockIdx.y;                      // chunk of 128 k = one quantization block
+    const int b = blockIdx.z;
+    const int k0 = kc * 128 + warp * 32 + khalf * 16;
+    const float* base = p.in + (int64_t)b * p.in_batch_stride + j;
+    const int64_t term_codes = (int64_t)p.rows * p.cols;
+
+    float raw[4][16];
+#pragma unroll
+    for (int jq = 0; jq < 4; ++jq)
+        if (jq < p.nq) {
+#pragma unroll
+            for (int kk = 0; kk < 16; ++kk)
+                raw[jq][kk] = __ldg(base + p.qoff[jq] + (int64_t)(k0 + kk) * p.ld);
+        }
+    auto combine = [&](int r, float (&v)[16]) {
+        bool set = false;
+#pragma unroll
+        for (int jq = 0; jq < 4; ++jq) {
+            const float cj = p.coef[r][jq];
+            if (coef_used<NZ>(r, jq, cj)) {
+                if (!set) {
+#pragma unroll
+                    for (int kk = 0; kk < 16; ++kk) v[kk] = __fmul_rn(cj, raw[jq][kk]);
+                    set = true;
+                } else {
+#pragma unroll
+                    for (int kk = 0; kk < 16; ++kk) v[kk] = __fmaf_rn(cj, raw[jq][kk], v[kk]);
+                }
+            }
+        }
+        if (!set) {
+#pragma unroll
+            for (int kk = 0; kk < 16; ++kk) v[kk] = 0.0f;
+        }
+    };
+#pragma unroll
+    for (int r = 0; r < FMM_MAX_RANK; ++r) {
+        if (row_used<NZ>(r, p.R)) {
+            float v[16];
+            combine(r, v);
+            float amax = 0.0f;
+#pragma unroll
+            for (int kk = 0; kk < 16; ++kk) amax = fmaxf(amax, fabsf(v[kk]));
+            amax = fmaxf(amax, __shfl_xor_sync(FULL, amax, 16));
+            if (khalf == 0) sub_amax[warp][r][col] = amax;
+        }
+    }
+    __syncthreads();
+#pragma unroll
+    for (int r = 0; r < FMM_MAX_RANK; ++r) {
+        if (row_used<NZ>(r, p.R)) {
+            const float amax = fmaxf(fmaxf(sub_amax[0][r][col], sub_amax[1][r][col]), fmaxf(sub_amax[2][r][col], sub_amax[3][r][col]));
+            float sc; uint32_t e8;
+            const float inv = block_scale<MODE>(amax, p.amax_floor, sc, e8);
+            const int64_t t = (int64_t)b * p.R + r;
+            if (warp == 0 && khalf == 0) store_b_scale<MODE>(p, t, r, j, kc, kc, sc, 0u, false);
+            float v[16];
+            combine(r, v);
+            uint32_t wv[4];
+#pragma unroll
+            for (int g = 0; g < 4; ++g)
+                wv[g] = pack4_e4m3(__fmul_rn(v[4 * g], inv), __fmul_rn(v[4 * g + 1], inv),
+                                   __fmul_rn(v[4 * g + 2], inv), __fmul_rn(v[4 * g + 3], inv));
+            uint8_t* qp = p.q_out + t * term_codes + (int64_t)j * p.rows + k0;
+            if (FMM_GUARD(p.guard, qp, 16, 1204)) *reinterpret_cast<uint4*>(qp) = make_uint4(wv[0], wv[1], wv[2], wv[3]);
         }
     }
 }
@@ -671,6 +762,16 @@ void launch_b(const EncodeParams& p, dim3 grid, cudaStream_t st)
         default: encode_b_kernel<BLK, MODE, 0u, false, false><<<grid, 128, 0, st>>>(p); return;
     }
 }
+void launch_b128(const EncodeParams& p, dim3 grid, cudaStream_t st)
+{
+    const uint32_t m = (p.nq == 4) ? coef_mask(p) : 0u;
+    switch (m) {
+#define X(M) case M: encode_b128_kernel<M><<<grid, 128, 0, st>>>(p); return;
+        FMM_KNOWN_MASKS(X)
+#undef X
+        default: encode_b128_kernel<0u><<<grid, 128, 0, st>>>(p); return;
+    }
+}
 template <int BLK, int MODE>
 void launch_a2(const EncodeParams& p, unsigned g, cudaStream_t st)
 {
@@ -735,7 +836,7 @@ fmm_status_t fmm_launch_encode_b(const EncodeParams& p, int blk, int mode, cudaS
         else launch_b_opt<false, true>(p, grid, st);
     } else if (mode == FMM_SCALE_FP32_AMAX_DIV_448) {
         if (blk == 32) launch_b<32, FMM_SCALE_FP32_AMAX_DIV_448>(p, grid, st);
-        else launch_b<128, FMM_SCALE_FP32_AMAX_DIV_448>(p, grid, st);
+        else { grid.x = (unsigned)(p.cols / 16); launch_b128(p, grid, st); }
     } else {
         launch_b<32, FMM_SCALE_UE8M0_CEIL>(p, grid, st);
     }
