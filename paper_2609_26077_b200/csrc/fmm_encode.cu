@@ -399,6 +399,85 @@ __global__ void __launch_bounds__(TILE ? 256 : 128, TILE ? 2 : 4) encode_b_kerne
     }
 }
 
+// B side, block 32, one 32-k block per warp: the four warps of a block take the four 32-k blocks of one 128-k chunk
+// of the same 16 columns (thread = 16 k of one column, lanes l and l+16 the two halves of a block), so every thread
+// issues all its loads at once and a chunk is spread over four warps instead of being walked by one.
+// Grid: (cols / 16, rows / 128, batch), 128 threads.
+template <int MODE, uint32_t NZ>
+__global__ void __launch_bounds__(128, 4) encode_b32_kernel(const EncodeParams p)
+{
+    constexpr unsigned FULL = 0xffffffffu;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int col = lane & 15, khalf = lane >> 4;
+    const int j = blockIdx.x * 16 + col;
+    const int kc = blockIdx.y;                      // chunk of 128 k
+    const int kb = kc * 4 + warp;                   // this warp's quantization block
+    const int b = blockIdx.z;
+    const int k0 = kb * 32 + khalf * 16;
+    const float* base = p.in + (int64_t)b * p.in_batch_stride + j;
+    const int64_t term_codes = (int64_t)p.rows * p.cols;
+
+    float raw[4][16];
+#pragma unroll
+    for (int jq = 0; jq < 4; ++jq)
+        if (jq < p.nq) {
+#pragma unroll
+            for (int kk = 0; kk < 16; ++kk)
+                raw[jq][kk] = __ldg(base + p.qoff[jq] + (int64_t)(k0 + kk) * p.ld);
+        }
+#pragma unroll
+    for (int r = 0; r < FMM_MAX_RANK; ++r) {
+        if (row_used<NZ>(r, p.R)) {
+            float v[16];
+            bool set = false;
+#pragma unroll
+            for (int jq = 0; jq < 4; ++jq) {
+                const float cj = p.coef[r][jq];
+                if (coef_used<NZ>(r, jq, cj)) {
+                    if (!set) {
+#pragma unroll
+                        for (int kk = 0; kk < 16; ++kk) v[kk] = __fmul_rn(cj, raw[jq][kk]);
+                        set = true;
+                    } else {
+#pragma unroll
+                        for (int kk = 0; kk < 16; ++kk) v[kk] = __fmaf_rn(cj, raw[jq][kk], v[kk]);
+                    }
+                }
+            }
+            if (!set) {
+#pragma unroll
+                for (int kk = 0; kk < 16; ++kk) v[kk] = 0.0f;
+            }
+            float amax = 0.0f;
+#pragma unroll
+            for (int kk = 0; kk < 16; ++kk) amax = fmaxf(amax, fabsf(v[kk]));
+            amax = fmaxf(amax, __shfl_xor_sync(FULL, amax, 16));
+            float sc; uint32_t e8;
+            const float inv = block_scale<MODE>(amax, p.amax_floor, sc, e8);
+            const int64_t t = (int64_t)b * p.R + r;
+            if (khalf == 0) {
+                char* so = reinterpret_cast<char*>(p.s_out) + t * p.s_term_stride;
+                const int jg = j + r * p.s_step;                   // column inside the scale array
+                if (MODE == FMM_SCALE_FP32_AMAX_DIV_448) {
+                    float* sp = reinterpret_cast<float*>(so) + (int64_t)kb * p.s_ld + jg;
+                    if (FMM_GUARD(p.guard, sp, 4, 1205)) *sp = sc;
+                } else {
+                    const int64_t tile = (int64_t)kc * p.sf_blocks + (jg >> 7);
+                    char* sp = so + tile * 512 + (jg & 31) * 16 + ((jg & 127) >> 5) * 4 + warp;
+                    if (FMM_GUARD(p.guard, sp, 1, 1206)) *reinterpret_cast<uint8_t*>(sp) = (uint8_t)e8;
+                }
+            }
+            uint32_t wv[4];
+#pragma unroll
+            for (int g = 0; g < 4; ++g)
+                wv[g] = pack4_e4m3(__fmul_rn(v[4 * g], inv), __fmul_rn(v[4 * g + 1], inv),
+                                   __fmul_rn(v[4 * g + 2], inv), __fmul_rn(v[4 * g + 3], inv));
+            uint8_t* qp = p.q_out + t * term_codes + (int64_t)j * p.rows + k0;
+            if (FMM_GUARD(p.guard, qp, 16, 1207)) *reinterpret_cast<uint4*>(qp) = make_uint4(wv[0], wv[1], wv[2], wv[3]);
+        }
+    }
+}
+
 // B side, block 128, per-column scales, one pass.  The four warps of a block take the four 32-k sub-blocks of one
 // 128-k block of the same 16 columns; every thread forms the combinations of its 16 k x 1 column, the sub-block
 // maxima meet in shared memory, and each warp then quantizes its own sub-block from the raw values it still holds
@@ -762,6 +841,17 @@ void launch_b(const EncodeParams& p, dim3 grid, cudaStream_t st)
         default: encode_b_kernel<BLK, MODE, 0u, false, false><<<grid, 128, 0, st>>>(p); return;
     }
 }
+template <int MODE>
+void launch_b32(const EncodeParams& p, dim3 grid, cudaStream_t st)
+{
+    const uint32_t m = (p.nq == 4) ? coef_mask(p) : 0u;
+    switch (m) {
+#define X(M) case M: encode_b32_kernel<MODE, M><<<grid, 128, 0, st>>>(p); return;
+        FMM_KNOWN_MASKS(X)
+#undef X
+        default: encode_b32_kernel<MODE, 0u><<<grid, 128, 0, st>>>(p); return;
+    }
+}
 void launch_b128(const EncodeParams& p, dim3 grid, cudaStream_t st)
 {
     const uint32_t m = (p.nq == 4) ? coef_mask(p) : 0u;
@@ -835,10 +925,12 @@ fmm_status_t fmm_launch_encode_b(const EncodeParams& p, int blk, int mode, cudaS
         else if (p.b_tile) launch_b_opt<true, false>(p, grid, st);
         else launch_b_opt<false, true>(p, grid, st);
     } else if (mode == FMM_SCALE_FP32_AMAX_DIV_448) {
-        if (blk == 32) launch_b<32, FMM_SCALE_FP32_AMAX_DIV_448>(p, grid, st);
-        else { grid.x = (unsigned)(p.cols / 16); launch_b128(p, grid, st); }
+        grid.x = (unsigned)(p.cols / 16);
+        if (blk == 32) launch_b32<FMM_SCALE_FP32_AMAX_DIV_448>(p, grid, st);
+        else launch_b128(p, grid, st);
     } else {
-        launch_b<32, FMM_SCALE_UE8M0_CEIL>(p, grid, st);
+        grid.x = (unsigned)(p.cols / 16);
+        launch_b32<FMM_SCALE_UE8M0_CEIL>(p, grid, st);
     }
     return cudaGetLastError() == cudaSuccess ? FMM_OK : FMM_ERR_CUDA;
 }

@@ -84,7 +84,6 @@ struct Cfg {
     static constexpr int SB_PART_BYTES = MX ? 0 : KB_PER_STAGE * BN * 4;
     static constexpr int SB_STAGE_BYTES = MX ? 0 : KB_PER_STAGE * (BN + BM) * 4;
     static constexpr int TX_BYTES = NCTA * (A_BYTES + B_BYTES + SF_STAGE_BYTES);
-    static constexpr int TX_BYTES_HALF = NCTA * (A_BYTES + B_BYTES / 2 + 1024);   // half-width item: one SFB atom
     static constexpr int OFF_A = 0;
     static constexpr int OFF_B = OFF_A + STAGES * A_BYTES;
     static constexpr int OFF_STG = OFF_B + STAGES * B_BYTES;
@@ -103,11 +102,6 @@ struct Cfg {
     static constexpr int ACC_BUFS = MX ? 1 : (512 / BN) / GPB;        // ring of (GPB x BN)-column super-buffers
     static constexpr int SF_COLS = 4 + 4 * SFB_ATOMS;
     static constexpr int CW = BN / 2;      // columns per epilogue warp
-    // Tail split (UE8M0, 256-column tiles): when the last wave of tile positions would occupy at most half
-    // of the CTAs (pairs), each of those positions is cut into two 128-column items, so the last wave
-    // takes about half as long.  Every item still runs all its terms in one CTA (pair): no output tile is
-    // shared between CTAs and the summation order stays fixed.
-    static constexpr bool SPLIT = MX && BN == 256;
     static_assert(SMEM_BYTES <= 232448, "shared memory budget");
     static_assert(!MX || BN + STAGES * SF_COLS <= 512, "TMEM budget");
 };
@@ -165,8 +159,9 @@ struct KParams {
     int m, n, k, terms;
     // Work items.  A slot is (term group, tile position): the terms of one group (the R products of one parent
     // at the innermost level; all terms at one level) feed one set of output blocks and are walked by one CTA
-    // (pair) in order.  Slots >= split_from are cut into two 128-column items.
-    int positions, terms_per_group, split_from, items;
+    // (pair) in order.  (Cutting the slots of a short last wave into narrower items does not pay: a tcgen05.mma of
+    // half the width takes as long to issue, measured 4 % slower at n = 8192.)
+    int positions, terms_per_group, items;
     const int* out_start; const FmmOutEntry* out;
     int* status;
     const float* c_base; long long ldc;       // the output matrix as plain memory: used by the FMM_DEBUG store guard only
@@ -177,8 +172,7 @@ template <int BN, int MODE, int BLK, int NCTA>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                 const __grid_constant__ CUtensorMap tmC, const __grid_constant__ CUtensorMap tmSFA,
-                const __grid_constant__ CUtensorMap tmSFB, const __grid_constant__ CUtensorMap tmBh,
-                const __grid_constant__ CUtensorMap tmSFBh, const KParams p)
+                const __grid_constant__ CUtensorMap tmSFB, const KParams p)
 {
     using C = Cfg<BN, MODE, BLK, NCTA>;
     extern __shared__ uint8_t smem_raw[];
@@ -224,10 +218,6 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     const uint32_t tmem_base = *tmem_slot;
 
     const int tiles_n = p.n / BN;
-    // work item w -> tile position, column offset inside the position, half-width flag
-    auto item_slot = [&](int w) { return (C::SPLIT && w >= p.split_from) ? p.split_from + ((w - p.split_from) >> 1) : w; };
-    auto item_half = [&](int w) { return C::SPLIT && w >= p.split_from; };
-    auto item_coff = [&](int w) { return (C::SPLIT && w >= p.split_from) ? ((w - p.split_from) & 1) * (BN / 2) : 0; };
     const int kstages = p.k / BK;
     const int nkb = p.k / BLK;
     const int row_blocks_a = p.m / 128, row_blocks_b = p.n / 128;
@@ -240,8 +230,7 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             int stage = 0; uint32_t phase = 0;
             bool ok = true;
             for (int w = unit; w < p.items && ok; w += units) {
-                const int slot = item_slot(w), coff = item_coff(w);
-                const bool half = item_half(w);
+                const int slot = w;
                 const int grp = slot / p.positions, pos = slot - grp * p.positions;
                 const int tm = pos / tiles_n, tn = pos % tiles_n;
                 const int row_blk = tm * NCTA + cta_rank;                 // 128-row block of S_r this CTA owns
@@ -251,22 +240,15 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                         if (!mbar_wait(bar_empty(stage), phase ^ 1u, ctl, 101)) { ok = false; break; }
                         // completion is counted on the even CTA's barrier; only that CTA arms it
                         const uint32_t fb = (NCTA == 2) ? (bar_full(stage) & PEER_BIT_MASK) : bar_full(stage);
-                        if (leader) mbar_expect_tx(bar_full(stage), half ? C::TX_BYTES_HALF : C::TX_BYTES);
+                        if (leader) mbar_expect_tx(bar_full(stage), C::TX_BYTES);
                         tma_load_2d<NCTA>(base + C::OFF_A + stage * C::A_BYTES, &tmA, ks * BK, t * p.m + row_blk * BM, fb);
-                        if (!half)
-                            tma_load_2d<NCTA>(base + C::OFF_B + stage * C::B_BYTES, &tmB, ks * BK,
-                                              t * p.n + tn * BN + cta_rank * C::BROWS, fb);
-                        else
-                            tma_load_2d<NCTA>(base + C::OFF_B + stage * C::B_BYTES, &tmBh, ks * BK,
-                                              t * p.n + tn * BN + coff + cta_rank * (C::BROWS / 2), fb);
+                        tma_load_2d<NCTA>(base + C::OFF_B + stage * C::B_BYTES, &tmB, ks * BK,
+                                          t * p.n + tn * BN + cta_rank * C::BROWS, fb);
                         if (C::MX) {
                             // scale tiles: 512-byte atoms, ordered [term][k quad][128-row block]
                             const uint32_t sf = base + C::OFF_SF + stage * C::SF_STAGE_BYTES;
                             tma_load_2d<NCTA>(sf, &tmSFA, 0, (t * (nkb >> 2) + ks) * row_blocks_a + row_blk, fb);
-                            if (!half)
-                                tma_load_2d<NCTA>(sf + 512, &tmSFB, 0, (t * (nkb >> 2) + ks) * row_blocks_b + tn * C::SFB_ATOMS, fb);
-                            else
-                                tma_load_2d<NCTA>(sf + 512, &tmSFBh, 0, (t * (nkb >> 2) + ks) * row_blocks_b + tn * C::SFB_ATOMS + coff / 128, fb);
+                            tma_load_2d<NCTA>(sf + 512, &tmSFB, 0, (t * (nkb >> 2) + ks) * row_blocks_b + tn * C::SFB_ATOMS, fb);
                         }
                         if (++stage == C::STAGES) { stage = 0; phase ^= 1u; }
                     }
@@ -281,7 +263,7 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             int ss = 0; uint32_t sphase = 0;
             bool ok = true;
             for (int w = unit; w < p.items && ok; w += units) {
-                const int slot = item_slot(w);
+                const int slot = w;
                 const int grp = slot / p.positions, pos = slot - grp * p.positions;
                 const int tn = pos % tiles_n;
                 const int t_end = (grp + 1) * p.terms_per_group;
@@ -311,7 +293,7 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             uint32_t dphase = 0, store_cnt = 0;
             bool ok = true;
             for (int w = unit; w < p.items && ok; w += units) {
-                const int slot = item_slot(w);
+                const int slot = w;
                 const int grp = slot / p.positions, pos = slot - grp * p.positions;
                 const int tm = pos / tiles_n, tn = pos % tiles_n;
                 const int t_end = (grp + 1) * p.terms_per_group;
@@ -389,9 +371,7 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             if (C::MX) idesc_full = (1u << 23) | ((uint32_t)(BN >> 3) << 17) | (MDIM << 24);
             else idesc_full = (1u << 4) | ((uint32_t)(BN >> 3) << 17) | (MDIM << 24);
             for (int w = unit; w < p.items && ok; w += units) {
-                const bool half = item_half(w);
-                // a half-width item is the same instruction with N = BN/2
-                const uint32_t idesc = half ? (idesc_full & ~(0x3Fu << 17)) | ((uint32_t)(BN >> 4) << 17) : idesc_full;
+                const uint32_t idesc = idesc_full;
                 for (int t = 0; t < p.terms_per_group && ok; ++t) {
                     if (C::MX) {
                         if (!mbar_wait_warp(bar_tempty(0), bphase ^ 1u, ctl, 201)) { ok = false; break; }
@@ -409,7 +389,7 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                             tc_cp_32x128b_warpx4<NCTA>(tsfa, make_sf_desc(sf));
 #pragma unroll
                             for (int h = 0; h < C::SFB_ATOMS; ++h)
-                                if (h == 0 || !half) tc_cp_32x128b_warpx4<NCTA>(tsfb + 4 * h, make_sf_desc(sf + 512 + h * 512));
+                                tc_cp_32x128b_warpx4<NCTA>(tsfb + 4 * h, make_sf_desc(sf + 512 + h * 512));
 #pragma unroll
                             for (int j = 0; j < BK / 32; ++j) {
                                 const uint32_t id = idesc | ((uint32_t)j << 29) | ((uint32_t)j << 4);
@@ -461,12 +441,12 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         uint32_t accu[C::MX ? C::CW : 1];               // UE8M0: raw fp32 bits drained from TMEM
         unsigned long long acc2[C::MX ? 1 : C::CW / 2]; // FP32: promoted accumulators, two columns per register pair
         for (int w = unit; w < p.items && ok; w += units) {
-            const int slot = item_slot(w), coff = item_coff(w);
+            const int slot = w;
             const int grp = slot / p.positions, pos = slot - grp * p.positions;
             const int tm = pos / tiles_n, tn = pos % tiles_n;
             const int row_in_leaf = (tm * NCTA + cta_rank) * BM + q * 32;
-            // columns this warp owns: half of the item's width, in 32-column chunks
-            const int cw = item_half(w) ? C::CW / 2 : C::CW;
+            // columns this warp owns, in 32-column chunks
+            constexpr int cw = C::CW;
             const int nch = cw / 32;
             const uint32_t lane_taddr = tmem_base + ((uint32_t)(q * 32) << 16) + h * cw;
             for (int t = grp * p.terms_per_group, left = p.terms_per_group; left > 0 && ok; ++t, --left) {
@@ -646,7 +626,7 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                 for (int o = o0; o < o1; ++o) {
                     const FmmOutEntry ent = p.out[o];
                     const int row0 = ent.row_off * p.m + row_in_leaf;
-                    const int col0 = ent.col_off * p.n + tn * BN + coff + h * cw;
+                    const int col0 = ent.col_off * p.n + tn * BN + h * cw;
 #pragma unroll
                     for (int c = 0; c < C::CW / C::CH; ++c) {
                         if (c * C::CH >= cw) break;
@@ -752,7 +732,7 @@ template <int BN, int MODE, int BLK, int NCTA>
 fmm_status_t launch(const GemmParams& g, cudaStream_t st)
 {
     using C = Cfg<BN, MODE, BLK, NCTA>;
-    CUtensorMap tmA, tmB, tmC, tmSFA, tmSFB, tmBh, tmSFBh;
+    CUtensorMap tmA, tmB, tmC, tmSFA, tmSFB;
     const CUtensorMapSwizzle SW = CU_TENSOR_MAP_SWIZZLE_128B;
     if (!make_map_2d(&tmA, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, g.qa, (uint64_t)g.k, (uint64_t)g.terms * g.m, BK, BM, SW)) return FMM_ERR_CUDA;
     if (!make_map_2d(&tmB, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, g.qb, (uint64_t)g.k, (uint64_t)g.terms * g.n, BK, C::BROWS, SW)) return FMM_ERR_CUDA;
@@ -765,13 +745,6 @@ fmm_status_t launch(const GemmParams& g, cudaStream_t st)
         if (!make_map_2d(&tmSFB, CU_TENSOR_MAP_DATA_TYPE_UINT32, 4, g.sb, 128, atoms_b, 128, C::SFB_ATOMS, CU_TENSOR_MAP_SWIZZLE_NONE)) return FMM_ERR_CUDA;
     } else {
         tmSFA = tmA; tmSFB = tmB;       // unused in this mode
-    }
-    tmBh = tmB; tmSFBh = tmSFB;
-    if (C::SPLIT) {
-        // half-width items: half as many rows of T_r per CTA, one scale atom
-        const uint64_t atoms_b = (uint64_t)g.terms * (g.k / 128) * (g.n / 128);
-        if (!make_map_2d(&tmBh, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, g.qb, (uint64_t)g.k, (uint64_t)g.terms * g.n, BK, C::BROWS / 2, SW)) return FMM_ERR_CUDA;
-        if (!make_map_2d(&tmSFBh, CU_TENSOR_MAP_DATA_TYPE_UINT32, 4, g.sb, 128, atoms_b, 128, 1, CU_TENSOR_MAP_SWIZZLE_NONE)) return FMM_ERR_CUDA;
     }
     int dev = 0, sms = 0;
     cudaGetDevice(&dev);
@@ -797,15 +770,12 @@ fmm_status_t launch(const GemmParams& g, cudaStream_t st)
     }
     const int slots = positions * (g.terms / tpg);
     const int units = slots < max_units ? slots : max_units;
-    const int tail = slots % units;
-    const bool split = C::SPLIT && tail > 0 && 2 * tail <= units;
     KParams kp;
     kp.sa = static_cast<const uint8_t*>(g.sa); kp.sb = static_cast<const uint8_t*>(g.sb);
     kp.sa_term = g.sa_term; kp.sb_term = g.sb_term;
     kp.m = g.m; kp.n = g.n; kp.k = g.k; kp.terms = g.terms;
     kp.positions = positions; kp.terms_per_group = tpg;
-    kp.split_from = split ? slots - tail : slots;
-    kp.items = slots + (split ? tail : 0);
+    kp.items = slots;
     kp.out_start = g.out_start; kp.out = g.out; kp.status = g.status;
     kp.c_base = g.C; kp.ldc = g.Nfull; kp.guard = g.guard;
 
@@ -819,7 +789,7 @@ fmm_status_t launch(const GemmParams& g, cudaStream_t st)
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = NCTA; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
-    cudaError_t ce = cudaLaunchKernelEx(&cfg, fmm_gemm_kernel<BN, MODE, BLK, NCTA>, tmA, tmB, tmC, tmSFA, tmSFB, tmBh, tmSFBh, kp);
+    cudaError_t ce = cudaLaunchKernelEx(&cfg, fmm_gemm_kernel<BN, MODE, BLK, NCTA>, tmA, tmB, tmC, tmSFA, tmSFB, kp);
     if (ce != cudaSuccess) { cudaGetLastError(); return FMM_ERR_CUDA; }
     return FMM_OK;
 }
