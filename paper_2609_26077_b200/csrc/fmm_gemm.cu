@@ -47,14 +47,18 @@ constexpr int EPI_WARPS = 8;               // two per TMEM lane quadrant, each h
 constexpr int EPI_WARP0 = 4;               // warps 0..3: operand producer, MMA issuer, scale producer (FP32 modes), idle
 constexpr int NUM_THREADS = (EPI_WARP0 + EPI_WARPS) * 32;
 // setmaxnreg budget: the CTA's register pool is NUM_THREADS x (registers at launch); an increase
-// beyond what the decrease freed would block forever, so the split is checked here.
-constexpr int REGS_AT_LAUNCH = 168, REGS_CTRL = 56, REGS_EPI = 224;
-static_assert(EPI_WARP0 * 32 * REGS_CTRL + EPI_WARPS * 32 * REGS_EPI <= NUM_THREADS * REGS_AT_LAUNCH, "register pool");
+// beyond what the decrease freed would block forever, so every split is checked (see Cfg).
+constexpr int REGS_AT_LAUNCH = 168;
 static_assert(NUM_THREADS * (REGS_AT_LAUNCH + 8) > 65536, "REGS_AT_LAUNCH must be the launch-bound maximum");
 
 template <int BN, int MODE, int BLK, int NCTA>
 struct Cfg {
     static constexpr bool MX = (MODE == FMM_SCALE_UE8M0_CEIL);
+    // Register split between the four control warps and the eight epilogue warps.  The FP32-scale kernels give the
+    // promoting warps all they can (accumulators + a TMEM chunk + scales); the UE8M0 kernel's epilogue needs less and
+    // its producer and issuer, which also handle the scale tiles, spilled at 56.
+    static constexpr int REGS_CTRL = MX ? 72 : 56, REGS_EPI = MX ? 208 : 224;
+    static_assert(EPI_WARP0 * 32 * REGS_CTRL + EPI_WARPS * 32 * REGS_EPI <= NUM_THREADS * REGS_AT_LAUNCH, "register pool");
     static constexpr int BROWS = BN / NCTA;                  // T_r rows this CTA loads per stage
     static constexpr int A_BYTES = BM * BK;
     static constexpr int B_BYTES = BROWS * BK;
@@ -223,7 +227,7 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     const int row_blocks_a = p.m / 128, row_blocks_b = p.n / 128;
 
     if (warp < EPI_WARP0) {
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(REGS_CTRL));
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(C::REGS_CTRL));
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
@@ -423,12 +427,11 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     }
     } else {
         // ------------------------------------------------------------------ epilogue warps
-        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(REGS_EPI));
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(C::REGS_EPI));
         const int e = warp - EPI_WARP0;
         const int q = warp & 3;            // TMEM lane quadrant this warp may access
         const int h = e >> 2;              // column half
         const uint32_t stg = base + C::OFF_STG + e * C::STAGING_BUFS * C::STAGING_BYTES;
-        uint8_t* stg_ptr = base_ptr + C::OFF_STG + e * C::STAGING_BUFS * C::STAGING_BYTES;
         // the accumulator-free signal goes to the MMA issuer, which lives in the even CTA
         auto release_acc = [&](int b) {
             if (NCTA == 2) mbar_arrive_cluster(bar_tempty(b) & PEER_BIT_MASK); else mbar_arrive(bar_tempty(b));
@@ -634,7 +637,7 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                         if (lane == 0) bulk_wait_read<C::STAGING_BUFS - 1>();   // the buffer about to be rewritten has been read
                         __syncwarp();
                         // one row of the chunk per lane; 16-byte pieces permuted as the tensor map's swizzle expects
-                        uint8_t* dst = stg_ptr + b * C::STAGING_BYTES + lane * (C::CH * 4);
+                        const uint32_t dst = stg + b * C::STAGING_BYTES + lane * (C::CH * 4);
                         const int swz = (C::CH == 32) ? (lane & 7) : ((lane >> 1) & 3);
                         if (C::ROWS4) {
                             // four-row layout: rows lane/4 + 8k, column pairs 8j + 2(lane%4) of this 32-column chunk
@@ -661,7 +664,7 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                                 unpack2(acc2[c * (C::CH / 2) + i4 * 2 + 1], v.z, v.w);
                             }
                             v.x *= ent.w; v.y *= ent.w; v.z *= ent.w; v.w *= ent.w;
-                            *reinterpret_cast<float4*>(dst + ((i4 ^ swz) << 4)) = v;
+                            sts128(dst + ((i4 ^ swz) << 4), v);
                         }
                         fence_proxy_async();
                         __syncwarp();

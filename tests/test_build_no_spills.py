@@ -1,6 +1,6 @@
-"""The product kernel's single-thread producer / issuer roles run with 56 registers after setmaxnreg; a few
-spilled values in their loops cost a quarter of the throughput of the balanced kernels.  Compile the file
-with ptxas statistics and require spill-free benchmark kernels and next to no spills elsewhere."""
+"""The product kernel's producer / issuer warps run with 56 or 72 registers after setmaxnreg; a few spilled values in
+their loops cost a quarter of the throughput of the balanced kernels.  Compile the file with ptxas statistics and
+require every instantiation to be spill-free."""
 import os
 import re
 import shutil
@@ -22,10 +22,7 @@ def test_product_kernel_has_no_register_spills():
     text = out.stderr + out.stdout
     entries = re.findall(r"Compiling entry function '([^']*fmm_gemm_kernel[^']*)'.*?\n.*?\n\s*(\d+) bytes stack frame, (\d+) bytes spill stores, (\d+) bytes spill loads", text)
     assert len(entries) >= 8, "ptxas statistics not found"
-    # the benchmark kernels (fp32 scales / block 32 with the output warp; UE8M0) must be spill-free; elsewhere a
-    # couple of spilled values (<= 32 bytes of spill stores) are tolerated, the damaging cases were larger
     bench = ("ILi128ELi3ELi32ELi2", "ILi256ELi1ELi32ELi2")
-    bad = [(name[-60:], st, ld) for name, _, st, ld in entries
-           if (any(b in name for b in bench) and (int(st) or int(ld))) or int(st) > 32]
+    bad = [(name[-60:], st, ld) for name, _, st, ld in entries if int(st) or int(ld)]
     assert not bad, f"register spills in {bad}"
     assert all(any(b in name for name, *_ in entries) for b in bench), "benchmark kernels not found"
