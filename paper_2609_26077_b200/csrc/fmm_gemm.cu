@@ -57,7 +57,7 @@ struct Cfg {
     // Register split between the four control warps and the eight epilogue warps.  The FP32-scale kernels give the
     // promoting warps all they can (accumulators + a TMEM chunk + scales); the UE8M0 kernel's epilogue needs less and
     // its producer and issuer, which also handle the scale tiles, spilled at 56.
-    static constexpr int REGS_CTRL = MX ? 72 : 56, REGS_EPI = MX ? 208 : 224;
+    static constexpr int REGS_CTRL = (MX || MODE == MODE_FP32_OUT_WARP) ? 72 : 56, REGS_EPI = (MX || MODE == MODE_FP32_OUT_WARP) ? 208 : 224;
     static_assert(EPI_WARP0 * 32 * REGS_CTRL + EPI_WARPS * 32 * REGS_EPI <= NUM_THREADS * REGS_AT_LAUNCH, "register pool");
     static constexpr int BROWS = BN / NCTA;                  // T_r rows this CTA loads per stage
     static constexpr int A_BYTES = BM * BK;
@@ -311,50 +311,54 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                         const FmmOutEntry ent = p.out[o];
                         const int row0 = ent.row_off * p.m + (tm * NCTA + cta_rank) * BM;
                         const int col0 = ent.col_off * p.n + tn * BN;
+                        // A weight of exactly 1 needs no copy: the promoting warps stored the chunks in the swizzled layout
+                        // the tensor map expects (and made them visible to the TMA engine), so they go out as they are.
+                        const bool direct = (ent.w == 1.0f);
 #pragma unroll 1
                         for (int ch0 = 0; ch0 < (BM / 32) * (BN / 32); ch0 += C::OUT_BUFS / 2) {
                             // OUT_BUFS/2 chunks of 32 rows x 32 columns per round (one proxy fence and one bulk group per
-                            // round, two rounds in flight).  The promoting warps stored the chunks in the swizzled layout
-                            // the tensor map expects; they are copied through registers to apply the weight.
+                            // round, two rounds in flight); other weights are applied on the way through registers.
                             const uint32_t b0 = (store_cnt & 1u) * (C::OUT_BUFS / 2);
-                            if (lane == 0) bulk_wait_read<1>();
-                            __syncwarp();
+                            if (!direct) {
+                                if (lane == 0) bulk_wait_read<1>();
+                                __syncwarp();
 #pragma unroll 1
-                            for (int k = 0; k < C::OUT_BUFS / 2; ++k) {
-                                const uint32_t src = dump + (ch0 + k) * 4096;
-                                const uint32_t dst = stg + (b0 + k) * 4096;
-#pragma unroll 1
-                                for (int i0 = 0; i0 < 8; i0 += 4) {      // four 16-byte pieces at a time: this warp has 56 registers
-                                    // same physical piece on both sides (the swizzle is kept); the lane-dependent order
-                                    // only spreads the 32 rows over the shared-memory banks.  All four loads are issued
-                                    // before the first store.
-                                    float4 v[4];
+                                for (int k = 0; k < C::OUT_BUFS / 2; ++k) {
+                                    const uint32_t src = dump + (ch0 + k) * 4096;
+                                    const uint32_t dst = stg + (b0 + k) * 4096;
+                                    // same physical piece on both sides (the swizzle is kept); the lane-dependent order only
+                                    // spreads the 32 rows over the shared-memory banks.  All loads are issued before the
+                                    // first store.
+                                    float4 v[8];
 #pragma unroll
-                                    for (int i4 = 0; i4 < 4; ++i4) v[i4] = lds128(src + (((i0 + i4) ^ (lane & 7)) << 4));
+                                    for (int i4 = 0; i4 < 8; ++i4) v[i4] = lds128(src + ((i4 ^ (lane & 7)) << 4));
 #pragma unroll
-                                    for (int i4 = 0; i4 < 4; ++i4) {
+                                    for (int i4 = 0; i4 < 8; ++i4) {
                                         v[i4].x *= ent.w; v[i4].y *= ent.w; v[i4].z *= ent.w; v[i4].w *= ent.w;
-                                        sts128(dst + (((i0 + i4) ^ (lane & 7)) << 4), v[i4]);
+                                        sts128(dst + ((i4 ^ (lane & 7)) << 4), v[i4]);
                                     }
                                 }
+                                fence_proxy_async();
+                                __syncwarp();
                             }
-                            fence_proxy_async();
-                            __syncwarp();
                             if (lane == 0) {
                                 const uint64_t pol_c = policy_evict_last();     // see the note on the C tiles' L2 policy below
+                                const uint32_t src0 = direct ? (base + C::OFF_DUMP + ch0 * 4096) : (base + C::OFF_STG + b0 * 4096);
 #pragma unroll 1
                                 for (int k = 0; k < C::OUT_BUFS / 2; ++k) {
                                     const int ch = ch0 + k;
                                     const int r = row0 + (ch / (BN / 32)) * 32, c = col0 + (ch % (BN / 32)) * 32;
                                     if (!FMM_GUARD(p.guard, p.c_base + (long long)r * p.ldc + c, (31 * p.ldc + 32) * 4, 1701)) continue;
-                                    if (ent.first) tma_store_2d_hint(&tmC, c, r, stg + (b0 + k) * 4096, pol_c);      // lane 0: stg = chunk base
-                                    else tma_reduce_add_2d_hint(&tmC, c, r, stg + (b0 + k) * 4096, pol_c);
+                                    if (ent.first) tma_store_2d_hint(&tmC, c, r, src0 + k * 4096, pol_c);
+                                    else tma_reduce_add_2d_hint(&tmC, c, r, src0 + k * 4096, pol_c);
                                 }
                                 bulk_commit();
                             }
-                            ++store_cnt;
+                            if (!direct) ++store_cnt;
                         }
                     }
+                    // the TMA engine has read the copy for the last time (chunks sent as they are), and so has every lane
+                    if (lane == 0) bulk_wait_read<0>();
                     // every lane has read the copy for the last time
                     __syncwarp();
                     if (lane == 0) mbar_arrive(bar_dempty);
@@ -613,6 +617,7 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                             sts64(dchunk + (j >> 2) * 4096 + rr * 128 + ((pc ^ (rr & 7)) << 4), acc2[k * 8 + j]);
                         }
                     }
+                    fence_proxy_async();          // the output warp may hand these chunks to the TMA engine as they are
                     __syncwarp();
                     if (lane == 0) mbar_arrive(bar_dfull);
                     continue;
@@ -805,16 +810,18 @@ fmm_status_t launch_shape(const GemmParams& g, cudaStream_t st)
     // on the CUDA cores and use 128-column tiles, whose four TMEM accumulators let the MMA issuer run
     // further ahead of the promoting warps.
     if constexpr (MODE != FMM_SCALE_UE8M0_CEIL) {
-        if constexpr (BLK == 128) {
-            // one promotion per 128 k: the tensor pipe matters again, and 256-column instructions read half as
-            // much shared memory per flop as 128-column ones
-            if ((g.m % 256) == 0 && (g.n % 256) == 0) return launch<256, MODE, BLK, 2>(g, st);
-        }
         if constexpr (BLK == 32 && MODE == FMM_SCALE_FP32_AMAX_DIV_448) {
-            if (g.k / BK >= 16) {           // long terms: post-addition by the output warp
+            // long terms: post-addition by the output warp.  (Block 128 does not gain from it: with 128-column tiles and
+            // the output warp it runs as fast as with 256-column tiles and none, 0.81 ms at n = 8192, and the cubic
+            // product, which has a single store per tile, is 20 % slower.)
+            if (g.k / BK >= 16) {
                 if ((g.m % 256) == 0) return launch<128, MODE_FP32_OUT_WARP, BLK, 2>(g, st);
                 return launch<128, MODE_FP32_OUT_WARP, BLK, 1>(g, st);
             }
+        }
+        if constexpr (BLK == 128) {
+            // one promotion per 128 k: 256-column tiles with two TMEM accumulators
+            if ((g.m % 256) == 0 && (g.n % 256) == 0) return launch<256, MODE, BLK, 2>(g, st);
         }
         if ((g.m % 256) == 0) return launch<128, MODE, BLK, 2>(g, st);
         return launch<128, MODE, BLK, 1>(g, st);
