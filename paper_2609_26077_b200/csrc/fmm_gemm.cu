@@ -230,7 +230,8 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(C::REGS_CTRL));
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
-        if (lane == 0) {
+        // (all lanes walk the loops, one elected lane issues: see the note on warp-collective issue in fmm_ptx.cuh)
+        {
             int stage = 0; uint32_t phase = 0;
             bool ok = true;
             for (int w = unit; w < p.items && ok; w += units) {
@@ -241,18 +242,20 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                 const int t_end = (grp + 1) * p.terms_per_group;
                 for (int t = t_end - p.terms_per_group; t < t_end && ok; ++t) {
                     for (int ks = 0; ks < kstages; ++ks) {
-                        if (!mbar_wait(bar_empty(stage), phase ^ 1u, ctl, 101)) { ok = false; break; }
+                        if (!mbar_wait_warp(bar_empty(stage), phase ^ 1u, ctl, 101)) { ok = false; break; }
                         // completion is counted on the even CTA's barrier; only that CTA arms it
                         const uint32_t fb = (NCTA == 2) ? (bar_full(stage) & PEER_BIT_MASK) : bar_full(stage);
-                        if (leader) mbar_expect_tx(bar_full(stage), C::TX_BYTES);
-                        tma_load_2d<NCTA>(base + C::OFF_A + stage * C::A_BYTES, &tmA, ks * BK, t * p.m + row_blk * BM, fb);
-                        tma_load_2d<NCTA>(base + C::OFF_B + stage * C::B_BYTES, &tmB, ks * BK,
-                                          t * p.n + tn * BN + cta_rank * C::BROWS, fb);
-                        if (C::MX) {
-                            // scale tiles: 512-byte atoms, ordered [term][k quad][128-row block]
-                            const uint32_t sf = base + C::OFF_SF + stage * C::SF_STAGE_BYTES;
-                            tma_load_2d<NCTA>(sf, &tmSFA, 0, (t * (nkb >> 2) + ks) * row_blocks_a + row_blk, fb);
-                            tma_load_2d<NCTA>(sf + 512, &tmSFB, 0, (t * (nkb >> 2) + ks) * row_blocks_b + tn * C::SFB_ATOMS, fb);
+                        if (elect_one()) {
+                            if (leader) mbar_expect_tx(bar_full(stage), C::TX_BYTES);
+                            tma_load_2d<NCTA>(base + C::OFF_A + stage * C::A_BYTES, &tmA, ks * BK, t * p.m + row_blk * BM, fb);
+                            tma_load_2d<NCTA>(base + C::OFF_B + stage * C::B_BYTES, &tmB, ks * BK,
+                                              t * p.n + tn * BN + cta_rank * C::BROWS, fb);
+                            if (C::MX) {
+                                // scale tiles: 512-byte atoms, ordered [term][k quad][128-row block]
+                                const uint32_t sf = base + C::OFF_SF + stage * C::SF_STAGE_BYTES;
+                                tma_load_2d<NCTA>(sf, &tmSFA, 0, (t * (nkb >> 2) + ks) * row_blocks_a + row_blk, fb);
+                                tma_load_2d<NCTA>(sf + 512, &tmSFB, 0, (t * (nkb >> 2) + ks) * row_blocks_b + tn * C::SFB_ATOMS, fb);
+                            }
                         }
                         if (++stage == C::STAGES) { stage = 0; phase ^= 1u; }
                     }
@@ -263,7 +266,7 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         // ------------------------------------------------------------------ FP32 modes: producer of the B-side scales
         // (its own thread and ring: the operand producer above has no registers to spare, and the scale ring is
         // released by the promoting warps, not by the tensor pipe)
-        if (!C::MX && lane == 0) {
+        if (!C::MX) {
             int ss = 0; uint32_t sphase = 0;
             bool ok = true;
             for (int w = unit; w < p.items && ok; w += units) {
@@ -276,14 +279,16 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                     const uint8_t* sb_t = p.sb + (long long)t * p.sb_term + (long long)tn * BN * 4;
                     const uint8_t* sa_t = p.sa + (long long)t * p.sa_term + (long long)(tm * NCTA + cta_rank) * BM * (C::KB_PER_STAGE * 4);
                     for (int ks = 0; ks < kstages; ++ks) {
-                        if (!mbar_wait(bar_sempty(ss), sphase ^ 1u, ctl, 102)) { ok = false; break; }
-                        mbar_expect_tx(bar_sfull(ss), C::SB_STAGE_BYTES);
+                        if (!mbar_wait_warp(bar_sempty(ss), sphase ^ 1u, ctl, 102)) { ok = false; break; }
+                        if (elect_one()) {
+                            mbar_expect_tx(bar_sfull(ss), C::SB_STAGE_BYTES);
 #pragma unroll
-                        for (int g = 0; g < C::KB_PER_STAGE; ++g)
-                            bulk_load(base + C::OFF_SB + ss * C::SB_STAGE_BYTES + g * BN * 4,
-                                      sb_t + (long long)(ks * C::KB_PER_STAGE + g) * p.n * 4, BN * 4, bar_sfull(ss));
-                        bulk_load(base + C::OFF_SB + ss * C::SB_STAGE_BYTES + C::SB_PART_BYTES,
-                                  sa_t + (long long)ks * p.m * (C::KB_PER_STAGE * 4), BM * C::KB_PER_STAGE * 4, bar_sfull(ss));
+                            for (int g = 0; g < C::KB_PER_STAGE; ++g)
+                                bulk_load(base + C::OFF_SB + ss * C::SB_STAGE_BYTES + g * BN * 4,
+                                          sb_t + (long long)(ks * C::KB_PER_STAGE + g) * p.n * 4, BN * 4, bar_sfull(ss));
+                            bulk_load(base + C::OFF_SB + ss * C::SB_STAGE_BYTES + C::SB_PART_BYTES,
+                                      sa_t + (long long)ks * p.m * (C::KB_PER_STAGE * 4), BM * C::KB_PER_STAGE * 4, bar_sfull(ss));
+                        }
                         if (++ss == C::SB_STAGES) { ss = 0; sphase ^= 1u; }
                     }
                 }
