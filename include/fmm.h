@@ -91,8 +91,10 @@ fmm_status_t fmm_plan_create(fmm_plan_t** plan, int rank, const float* U, const 
 fmm_status_t fmm_plan_destroy(fmm_plan_t* plan);
 
 /* Bytes of device workspace fmm_matmul / fmm_encode_only need for this problem size (host call).
- * The workspace holds the quantized leaf operands, their scales and, for levels >= 2, the fp32
- * intermediate combinations of the outer levels and the partially decoded products. */
+ * The workspace holds what the fused regime of Sec. 2.2 / App. D.1 produces between its steps: the quantized
+ * encoded combinations x_r, y_r of the R^levels leaves (e4m3 codes + one scale per block, App. E.2) and, for
+ * levels >= 2, the fp32 combinations of the outer levels and the partially decoded products of the level-by-level
+ * recursion (Sec. 3).  Never the products M_r themselves: those go from the tensor cores straight into C. */
 fmm_status_t fmm_workspace_bytes(const fmm_plan_t* plan, int64_t M, int64_t N, int64_t K,
                                  size_t* bytes);
 
@@ -128,18 +130,22 @@ fmm_status_t fmm_matmul_host(const fmm_plan_t* plan, const float* A, const float
                              int64_t M, int64_t N, int64_t K, void* workspace, size_t workspace_bytes,
                              void* cuda_stream);
 
-/* Steps 1-2 only (pre-addition + quantization of both sides) into the workspace. */
+/* The encoder alone (Sec. 2.1: x_r = <U_r, a>, y_r = <V_r, b>, formed in fp32 from the unquantized blocks; Sec. 2.2 /
+ * App. D.1: quantized only afterwards; App. E.2: scale and cast per block) for both sides, into the workspace.
+ * Arguments, shape rule and errors as fmm_matmul; C is not touched. */
 fmm_status_t fmm_encode_only(const fmm_plan_t* plan, const float* A, const float* B,
                              int64_t M, int64_t N, int64_t K, void* workspace,
                              size_t workspace_bytes, void* cuda_stream);
 
-/* The tensor-core products + post-addition only, on operands a previous fmm_encode_only /
- * fmm_matmul left in the workspace. */
+/* The products and the decoder alone (Sec. 2.1: c = sum_r (x_r^ y_r^) W_r, fp32 accumulation) on operands a previous
+ * fmm_encode_only / fmm_matmul left in the workspace.  Arguments, shape rule and errors as fmm_matmul. */
 fmm_status_t fmm_multiply_only(const fmm_plan_t* plan, float* C, int64_t M, int64_t N, int64_t K,
                                void* workspace, size_t workspace_bytes, void* cuda_stream);
 
-/* Where the quantized leaf operand of term `term` (depth-first order t = (r1*R + r2)*R + ...,
- * r1 = outermost level; 0 for levels == 0) lives in the workspace (host call, byte offsets).
+/* Where the quantized encoded combination (App. E.2: e4m3 codes and one scale per block of block_k elements along
+ * the contracted axis) of term `term` (depth-first order t = (r1*R + r2)*R + ..., the Kronecker order of Sec. 3;
+ * r1 = outermost level; 0 for levels == 0) lives in the workspace (host call, byte offsets).  This is the view the
+ * bit-parity tests read.
  *   side 'A': codes are q_rows x q_cols = (M/d) x (K/d) e4m3 bytes, row-major (K contiguous).
  *   side 'B': codes are stored TRANSPOSED, q_rows x q_cols = (N/d) x (K/d) (K contiguous).
  *   FP32 scale mode: fp32 scales, laid out as the product kernel fetches them per 128-k pipeline stage.
@@ -185,7 +191,8 @@ fmm_status_t fmm_error_stats_noalloc(const float* C, const double* Cref, int64_t
                                      double* out3, void* cuda_stream);
 int64_t fmm_error_stats_noalloc_max_elements(void);
 
-/* Reads the plan's device status word after cudaDeviceSynchronize (all streams of the device, non-blocking
+/* (No counterpart in the paper: failure reporting of this implementation.)
+ * Reads the plan's device status word after cudaDeviceSynchronize (all streams of the device, non-blocking
  * ones included, have drained).  *code == 0: no bounded wait has
  * given up since plan creation; otherwise a kernel-specific location code, and the results of the
  * call that set it are invalid.  Returns FMM_ERR_DEVICE_TIMEOUT when *code != 0. */
