@@ -212,6 +212,10 @@ fmm_status_t multiply(const fmm_plan* plan, const FmmLayout& L, char* ws, float*
     g.m = (int)L.m; g.n = (int)L.n; g.k = (int)L.k; g.terms = (int)L.terms;
     g.terms_per_group = plan->levels >= 2 ? plan->rank : (int)L.terms;
     g.out_start = plan->d_out_start; g.out = plan->d_out; g.status = plan->d_status;
+    g.pair_start = plan->d_pair_start; g.pair = plan->d_pair; g.steps = plan->steps;
+    // the pair-fused walk order belongs to the UE8M0 kernel; the fp32-scale kernels keep the products in term order
+    for (int r = 0; r < FMM_MAX_RANK; ++r)
+        g.order[r] = (plan->qp.scale_mode == FMM_SCALE_UE8M0_CEIL && plan->levels >= 1) ? plan->order[r] : r;
     g.sb_tile = plan->qp.b_tile_n == 128 ? 1 : 0;
     g.guard = fmm_make_guard(dest, (size_t)g.Mfull * (size_t)g.Nfull * 4, nullptr, 0, plan->d_status + FMM_GUARD_WORD);
     fmm_status_t s = fmm_launch_gemm(g, plan->qp.block_k, (int)plan->qp.scale_mode, st, launches);
@@ -344,6 +348,69 @@ fmm_status_t fmm_plan_create(fmm_plan_t** out, int rank, const float* U, const f
     start[p->terms] = (int)entries.size();
     p->n_out_total = (int)entries.size();
 
+    // Pair-fused decoder: pair up the R products of a parent so that the pairs' unions of destination blocks are as
+    // small as possible in total (exhaustive over the matchings: R <= 8), walk the pairs one after the other.
+    for (int r = 0; r < FMM_MAX_RANK; ++r) p->order[r] = r;
+    p->steps = levels >= 1 ? (rank + 1) / 2 : 1;
+    std::vector<int> pstart;
+    std::vector<FmmPairEntry> pentries;
+    if (levels >= 1) {
+        auto mask = [&](int r) { int m = 0; for (int q = 0; q < 4; ++q) if (p->W[r][q] != 0.0f) m |= 1 << q; return m; };
+        auto bits = [](int m) { return (m & 1) + ((m >> 1) & 1) + ((m >> 2) & 1) + ((m >> 3) & 1); };
+        int best_cost = 1 << 30, best[FMM_MAX_RANK], cur[FMM_MAX_RANK];
+        bool used[FMM_MAX_RANK] = {false};
+        // recursive matching: always pair the lowest unused product with some other one (or leave it single once)
+        struct Rec {
+            static void go(int n, int R, int cost, bool single_used, bool* used, int* cur, int& best_cost, int* best,
+                           const int* masks, int (*bitsf)(int))
+            {
+                if (cost >= best_cost) return;
+                int a = -1;
+                for (int r = 0; r < R; ++r) if (!used[r]) { a = r; break; }
+                if (a < 0) { best_cost = cost; for (int i = 0; i < R; ++i) best[i] = cur[i]; return; }
+                used[a] = true;
+                for (int b = a + 1; b < R; ++b) {
+                    if (used[b]) continue;
+                    used[b] = true; cur[n] = a; cur[n + 1] = b;
+                    go(n + 2, R, cost + bitsf(masks[a] | masks[b]), single_used, used, cur, best_cost, best, masks, bitsf);
+                    used[b] = false;
+                }
+                if ((R & 1) && !single_used) {
+                    // the single product goes last in the walk: remember it at the end of cur
+                    cur[R - 1] = a;
+                    // shift: pairs fill cur[0 .. R-2]
+                    go(n, R, cost + bitsf(masks[a]), true, used, cur, best_cost, best, masks, bitsf);
+                }
+                used[a] = false;
+            }
+        };
+        int masks[FMM_MAX_RANK];
+        for (int r = 0; r < rank; ++r) masks[r] = mask(r);
+        Rec::go(0, rank, 0, false, used, cur, best_cost, best, masks, +bits);
+        for (int r = 0; r < rank; ++r) p->order[r] = best[r];
+        std::vector<char> ptouched((size_t)parents * 4, 0);
+        for (int parent = 0; parent < parents; ++parent)
+            for (int s = 0; s < p->steps; ++s) {
+                pstart.push_back((int)pentries.size());
+                const bool pairstep = 2 * s + 1 < rank;
+                const int ra = pairstep ? p->order[2 * s] : -1, rb = pairstep ? p->order[2 * s + 1] : p->order[2 * s];
+                for (int q = 0; q < 4; ++q) {
+                    const float wa = ra >= 0 ? p->W[ra][q] : 0.0f, wb = p->W[rb][q];
+                    if (wa == 0.0f && wb == 0.0f) continue;
+                    FmmPairEntry e;
+                    e.row_off = parent * 2 + (q >> 1); e.col_off = q & 1; e.wA = wa; e.wB = wb;
+                    e.first = ptouched[(size_t)parent * 4 + q] ? 0 : 1;
+                    ptouched[(size_t)parent * 4 + q] = 1;
+                    pentries.push_back(e);
+                }
+            }
+    } else {
+        pstart.push_back(0);
+        FmmPairEntry e; e.row_off = 0; e.col_off = 0; e.wA = 0.0f; e.wB = 1.0f; e.first = 1;
+        pentries.push_back(e);
+    }
+    pstart.push_back((int)pentries.size());
+
     cudaError_t ce = cudaMalloc(&p->d_status, 64 * sizeof(int));
     if (ce == cudaSuccess) ce = cudaMalloc(&p->d_out_start, sizeof(int) * start.size());
     if (ce == cudaSuccess) ce = cudaMalloc(&p->d_out, sizeof(FmmOutEntry) * (entries.size() + 1));
@@ -351,6 +418,10 @@ fmm_status_t fmm_plan_create(fmm_plan_t** out, int rank, const float* U, const f
     if (ce == cudaSuccess) ce = cudaMemcpy(p->d_out_start, start.data(), sizeof(int) * start.size(), cudaMemcpyHostToDevice);
     if (ce == cudaSuccess && !entries.empty())
         ce = cudaMemcpy(p->d_out, entries.data(), sizeof(FmmOutEntry) * entries.size(), cudaMemcpyHostToDevice);
+    if (ce == cudaSuccess) ce = cudaMalloc(&p->d_pair_start, sizeof(int) * pstart.size());
+    if (ce == cudaSuccess) ce = cudaMalloc(&p->d_pair, sizeof(FmmPairEntry) * (pentries.size() + 1));
+    if (ce == cudaSuccess) ce = cudaMemcpy(p->d_pair_start, pstart.data(), sizeof(int) * pstart.size(), cudaMemcpyHostToDevice);
+    if (ce == cudaSuccess) ce = cudaMemcpy(p->d_pair, pentries.data(), sizeof(FmmPairEntry) * pentries.size(), cudaMemcpyHostToDevice);
     if (ce != cudaSuccess) {
         cudaGetLastError();
         fmm_plan_destroy(p);
@@ -366,6 +437,8 @@ fmm_status_t fmm_plan_destroy(fmm_plan_t* p)
     if (p->d_status) cudaFree(p->d_status);
     if (p->d_out_start) cudaFree(p->d_out_start);
     if (p->d_out) cudaFree(p->d_out);
+    if (p->d_pair_start) cudaFree(p->d_pair_start);
+    if (p->d_pair) cudaFree(p->d_pair);
     delete p;
     return FMM_OK;
 }

@@ -107,9 +107,16 @@ struct Cfg {
     static constexpr int GPB = MX ? 1 : ((KB_PER_STAGE >= 2 && 512 / BN >= 4) ? 2 : 1);
     static constexpr int ACC_BUFS = MX ? 1 : (512 / BN) / GPB;        // ring of (GPB x BN)-column super-buffers
     static constexpr int SF_COLS = 4 + 4 * SFB_ATOMS;
+    // UE8M0: TMEM columns [0, BN) accumulator, [BN, BN + SF_COLS) the scale factors of the stage being multiplied (one
+    // slot: tcgen05.cp and tcgen05.mma execute in issue order), then the HOLD area of the pair-fused decoder: every
+    // epilogue warp parks CW - 16 columns of a finished product there (the other 16 stay in registers) until the
+    // product it is paired with is done.
+    static constexpr int HOLD_T = MX ? (BN / 2 - 16) : 0;          // parked columns per warp
+    static constexpr int OFF_HOLD = BN + 16;
     static constexpr int CW = BN / 2;      // columns per epilogue warp
     static_assert(SMEM_BYTES <= 232448, "shared memory budget");
-    static_assert(!MX || BN + STAGES * SF_COLS <= 512, "TMEM budget");
+    static_assert(!MX || (SF_COLS <= 16 && OFF_HOLD + 2 * HOLD_T <= 512), "TMEM budget");
+    static_assert(!MX || HOLD_T == 112 || HOLD_T == 48, "hold area is parked with 32- and 16-column stores");
 };
 
 constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;   // 2 s: far beyond any legitimate wait
@@ -169,6 +176,8 @@ struct KParams {
     // half the width takes as long to issue, measured 4 % slower at n = 8192.)
     int positions, terms_per_group, items;
     const int* out_start; const FmmOutEntry* out;
+    const int* pair_start; const FmmPairEntry* pair;   // pair-fused decoder (UE8M0): steps of two products, see FmmPairEntry
+    int order[FMM_MAX_RANK]; int steps; int R;         // walk order of the R products of a parent; steps = ceil(R / 2)
     int* status;
     const float* c_base; long long ldc;       // the output matrix as plain memory: used by the FMM_DEBUG store guard only
     FmmGuard guard;
@@ -226,6 +235,9 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     const int tiles_n = p.n / BN;
     const int kstages = p.k / BK;
     const int nkb = p.k / BLK;
+    // ti-th product a CTA (pair) walks in work-item group grp: the parents of the group one after the other, the R
+    // products of a parent in the plan's walk order (identity unless the decoder is pair-fused)
+    auto term_of = [&](int grp, int ti) { return grp * p.terms_per_group + (ti / p.R) * p.R + p.order[ti % p.R]; };
     const int row_blocks_a = p.m / 128, row_blocks_b = p.n / 128;
 
     if (warp < EPI_WARP0) {
@@ -241,8 +253,8 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                 const int grp = slot / p.positions, pos = slot - grp * p.positions;
                 const int tm = pos / tiles_n, tn = pos % tiles_n;
                 const int row_blk = tm * NCTA + cta_rank;                 // 128-row block of S_r this CTA owns
-                const int t_end = (grp + 1) * p.terms_per_group;
-                for (int t = t_end - p.terms_per_group; t < t_end && ok; ++t) {
+                for (int ti = 0; ti < p.terms_per_group && ok; ++ti) {
+                    const int t = term_of(grp, ti);
                     for (int ks = 0; ks < kstages; ++ks) {
                         if (!mbar_wait_warp(bar_empty(stage), phase ^ 1u, ctl, 101)) { ok = false; break; }
                         // completion is counted on the even CTA's barrier; only that CTA arms it
@@ -399,7 +411,7 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                         const uint64_t bdesc = make_kmajor_sw128_desc(base + C::OFF_B + stage * C::B_BYTES);
                         if (C::MX) {
                             const uint32_t sf = base + C::OFF_SF + stage * C::SF_STAGE_BYTES;
-                            const uint32_t tsfa = tmem_base + BN + stage * C::SF_COLS;
+                            const uint32_t tsfa = tmem_base + BN;          // one slot: cp and mma execute in issue order
                             const uint32_t tsfb = tsfa + 4;
                             tc_cp_32x128b_warpx4<NCTA>(tsfa, make_sf_desc(sf));
 #pragma unroll
@@ -453,6 +465,7 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         uint32_t dphase = 0;
         bool ok = true;
         uint32_t accu[C::MX ? C::CW : 1];               // UE8M0: raw fp32 bits drained from TMEM
+        uint32_t kept[C::MX ? 16 : 1];                  // ... and the 16 columns of a parked product that stay in registers
         unsigned long long acc2[C::MX ? 1 : C::CW / 2]; // FP32: promoted accumulators, two columns per register pair
         for (int w = unit; w < p.items && ok; w += units) {
             const int slot = w;
@@ -463,7 +476,8 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             constexpr int cw = C::CW;
             const int nch = cw / 32;
             const uint32_t lane_taddr = tmem_base + ((uint32_t)(q * 32) << 16) + h * cw;
-            for (int t = grp * p.terms_per_group, left = p.terms_per_group; left > 0 && ok; ++t, --left) {
+            for (int ti = 0; ti < p.terms_per_group && ok; ++ti) {
+                const int t = term_of(grp, ti);
                 if (C::MX) {
                     if (!mbar_wait_warp(bar_tfull(0), bphase, ctl, 301)) { ok = false; break; }
                     tc_fence_after();
@@ -475,6 +489,73 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                     __syncwarp();
                     if (lane == 0) release_acc(0);
                     bphase ^= 1u;
+                    // ---- pair-fused post-addition (see FmmPairEntry).  First product of a step: park it - CW - 16
+                    // columns in this warp's part of the TMEM hold area, 16 in registers - and go on to the next product.
+                    const int ri = ti % p.R;
+                    const uint32_t hold_taddr = tmem_base + ((uint32_t)(q * 32) << 16) + C::OFF_HOLD + h * C::HOLD_T;
+                    if ((ri & 1) == 0 && ri + 1 < p.R) {
+#pragma unroll
+                        for (int c = 0; c < C::HOLD_T / 32; ++c) tmem_st32(hold_taddr + c * 32, &accu[c * 32]);
+                        tmem_st16(hold_taddr + (C::HOLD_T / 32) * 32, &accu[(C::HOLD_T / 32) * 32]);
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) kept[i] = accu[C::HOLD_T + i];
+                        tmem_st_wait();
+                        continue;
+                    }
+                    // second product of a step, or an unpaired one: one weighted update per destination block
+                    const uint64_t pol_c = policy_evict_last();
+                    const int sidx = (t / p.R) * p.steps + (ri >> 1);
+                    const int o0 = p.pair_start[sidx], o1 = p.pair_start[sidx + 1];
+                    if (lane == 0) bulk_wait<0>();     // the previous step's writes to these tiles have landed
+                    __syncwarp();
+                    for (int o = o0; o < o1; ++o) {
+                        const FmmPairEntry ent = p.pair[o];
+                        const int row0 = ent.row_off * p.m + row_in_leaf;
+                        const int col0 = ent.col_off * p.n + tn * BN + h * cw;
+                        const bool useA = (ent.wA != 0.0f);
+#pragma unroll
+                        for (int c = 0; c < C::CW / C::CH; ++c) {
+                            const uint32_t b = store_cnt & (C::STAGING_BUFS - 1);
+                            if (lane == 0) bulk_wait_read<C::STAGING_BUFS - 1>();   // the buffer about to be rewritten has been read
+                            __syncwarp();
+                            const uint32_t dst = stg + b * C::STAGING_BYTES + lane * (C::CH * 4);
+                            const int swz = (C::CH == 32) ? (lane & 7) : ((lane >> 1) & 3);
+#pragma unroll
+                            for (int s16 = 0; s16 < C::CH / 16; ++s16) {
+                                const int col = c * C::CH + s16 * 16;          // first of 16 columns, within this warp's CW
+                                uint32_t av[16];
+                                if (useA) {
+                                    if (col < C::HOLD_T) { tmem_ld16(hold_taddr + col, av); tmem_ld_wait(); }
+                                    else {
+#pragma unroll
+                                        for (int i = 0; i < 16; ++i) av[i] = kept[i];
+                                    }
+                                }
+#pragma unroll
+                                for (int i4 = 0; i4 < 4; ++i4) {
+                                    float4 v;
+                                    v.x = __uint_as_float(accu[col + i4 * 4 + 0]) * ent.wB; v.y = __uint_as_float(accu[col + i4 * 4 + 1]) * ent.wB;
+                                    v.z = __uint_as_float(accu[col + i4 * 4 + 2]) * ent.wB; v.w = __uint_as_float(accu[col + i4 * 4 + 3]) * ent.wB;
+                                    if (useA) {
+                                        v.x = fmaf(__uint_as_float(av[i4 * 4 + 0]), ent.wA, v.x); v.y = fmaf(__uint_as_float(av[i4 * 4 + 1]), ent.wA, v.y);
+                                        v.z = fmaf(__uint_as_float(av[i4 * 4 + 2]), ent.wA, v.z); v.w = fmaf(__uint_as_float(av[i4 * 4 + 3]), ent.wA, v.w);
+                                    }
+                                    sts128(dst + (((s16 * 4 + i4) ^ swz) << 4), v);
+                                }
+                            }
+                            fence_proxy_async();
+                            __syncwarp();
+                            if (lane == 0) {
+                                if (FMM_GUARD(p.guard, p.c_base + (long long)row0 * p.ldc + col0 + c * C::CH, (31 * p.ldc + C::CH) * 4, 1703)) {
+                                    if (ent.first) tma_store_2d_hint(&tmC, col0 + c * C::CH, row0, stg + b * C::STAGING_BYTES, pol_c);
+                                    else tma_reduce_add_2d_hint(&tmC, col0 + c * C::CH, row0, stg + b * C::STAGING_BYTES, pol_c);
+                                }
+                                bulk_commit();
+                            }
+                            ++store_cnt;
+                        }
+                    }
+                    continue;
                 } else if (C::ROWS4) {
                     // ---- per-column fp32 scales.  The accumulators are read with the
                     // 16-lane load shape: a thread owns four rows (lane/4 + 8k) x CW/4 columns (8j + 2(lane%4), +1)
@@ -792,6 +873,9 @@ fmm_status_t launch(const GemmParams& g, cudaStream_t st)
     kp.positions = positions; kp.terms_per_group = tpg;
     kp.items = slots;
     kp.out_start = g.out_start; kp.out = g.out; kp.status = g.status;
+    kp.pair_start = g.pair_start; kp.pair = g.pair; kp.steps = g.steps;
+    for (int r = 0; r < FMM_MAX_RANK; ++r) kp.order[r] = g.order[r];
+    kp.R = g.terms_per_group > 0 ? g.terms_per_group : 1;       // products per parent (1 for the cubic product)
     kp.c_base = g.C; kp.ldc = g.Nfull; kp.guard = g.guard;
 
     cudaLaunchConfig_t cfg;

@@ -50,6 +50,17 @@ static inline FmmGuard fmm_make_guard(const void* a, size_t na, const void* b, s
 // status word that receives guard violations: plan->d_status[FMM_GUARD_WORD]
 #define FMM_GUARD_WORD 2
 
+// Pair-fused decoder (UE8M0 product kernel): the R products of a parent are walked in an order in which consecutive
+// products (2s, 2s+1) form a step; the epilogue keeps product A on chip until product B is done and sends ONE weighted
+// update wA * M_A + wB * M_B to every output block either of them feeds, which cuts the number of block updates that
+// go through L2 (18 -> 11 for the Phi-optimal realization, 12 -> 9 for Strassen).  An unpaired last product is a step
+// with wA = 0.
+struct FmmPairEntry {
+    int row_off, col_off;     // destination block, in units of leaf blocks
+    float wA, wB;             // weights of the step's first and second product (wA = 0: first product absent / not used)
+    int first;                // 1: overwrite, 0: add
+};
+
 struct FmmLayout {            // byte offsets into the workspace
     int64_t m, n, k;          // leaf dimensions
     int64_t terms;            // R^levels (1 for levels == 0)
@@ -72,6 +83,10 @@ struct fmm_plan {
     int* d_out_start;         // [terms + 1]
     FmmOutEntry* d_out;       // [total entries], block offsets in units of leaf blocks (scaled at launch)
     int n_out_total;
+    int order[FMM_MAX_RANK];  // walk order of the R products of a parent (identity unless the decoder is pair-fused)
+    int steps;                // pair-fused decoder: steps per parent, ceil(R / 2)
+    int* d_pair_start;        // [parents * steps + 1]
+    FmmPairEntry* d_pair;     // entries of all steps
     // kernels launched by the most recent call on this plan; written once, at the end of a call (calls take the
     // plan as const, and two host threads may share one)
     mutable std::atomic<int> last_launches;
@@ -134,6 +149,8 @@ struct GemmParams {
     int64_t Mfull, Nfull;
     int m, n, k, terms;
     const int* out_start; const FmmOutEntry* out;
+    const int* pair_start; const FmmPairEntry* pair;   // pair-fused decoder tables (UE8M0 kernel)
+    int order[FMM_MAX_RANK]; int steps;
     int* status;
     int terms_per_group;                    // consecutive terms that feed the same output blocks (R at levels >= 2, else all)
     int sb_tile;                            // fp32 scales, blk 128: the B-side scale is constant over each 128-column tile
