@@ -865,7 +865,10 @@ fmm_status_t launch(const GemmParams& g, cudaStream_t st)
         if (many >= one) tpg = g.terms;
     }
     const int slots = positions * (g.terms / tpg);
-    const int units = slots < max_units ? slots : max_units;
+    // as few CTAs (pairs) as finish in the same number of waves: every unit then gets the same number of items, and
+    // fewer units contend for L2 (256 positions: 64 pairs in 4 waves instead of 74 pairs with a ragged fourth wave)
+    const int waves = (slots + max_units - 1) / max_units;
+    const int units = (slots + waves - 1) / waves;
     KParams kp;
     kp.sa = static_cast<const uint8_t*>(g.sa); kp.sb = static_cast<const uint8_t*>(g.sb);
     kp.sa_term = g.sa_term; kp.sb_term = g.sb_term;
