@@ -237,7 +237,10 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     const int nkb = p.k / BLK;
     // ti-th product a CTA (pair) walks in work-item group grp: the parents of the group one after the other, the R
     // products of a parent in the plan's walk order (identity unless the decoder is pair-fused)
-    auto term_of = [&](int grp, int ti) { return grp * p.terms_per_group + (ti / p.R) * p.R + p.order[ti % p.R]; };
+    auto term_of = [&](int grp, int ti) {
+        if constexpr (C::MX) return grp * p.terms_per_group + (ti / p.R) * p.R + p.order[ti % p.R];
+        else return grp * p.terms_per_group + ti;
+    };
     const int row_blocks_a = p.m / 128, row_blocks_b = p.n / 128;
 
     if (warp < EPI_WARP0) {
@@ -476,8 +479,8 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             constexpr int cw = C::CW;
             const int nch = cw / 32;
             const uint32_t lane_taddr = tmem_base + ((uint32_t)(q * 32) << 16) + h * cw;
-            for (int ti = 0; ti < p.terms_per_group && ok; ++ti) {
-                const int t = term_of(grp, ti);
+            for (int ti = 0, left = p.terms_per_group; left > 0 && ok; ++ti, --left) {
+                const int t = C::MX ? term_of(grp, ti) : grp * p.terms_per_group + ti;
                 if (C::MX) {
                     if (!mbar_wait_warp(bar_tfull(0), bphase, ctl, 301)) { ok = false; break; }
                     tc_fence_after();
