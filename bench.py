@@ -151,6 +151,14 @@ def combined_roofline_ms(M, N, K, levels, rank, mode, blk, fp8_peak_tflops, hbm_
     return (flops / (fp8_peak_tflops * 1e12) + (enc_bytes + gemm_bytes) / (hbm_gbs * 1e9)) * 1e3
 
 
+def overlap_bound_ms(M, N, K, levels, rank, mode, blk, fp8_peak_tflops, hbm_gbs):
+    """The same two terms with the phases fully overlapped: max(tensor time, HBM time).  No schedule of this path
+    can reach it (the products need the encoded operands), it brackets the serialized roofline from below."""
+    scale_bytes = 1 if mode.startswith("ue8m0") else 4
+    flops, enc_bytes, gemm_bytes = algorithmic_work(M, N, K, levels, rank, scale_bytes, blk)
+    return max(flops / (fp8_peak_tflops * 1e12), (enc_bytes + gemm_bytes) / (hbm_gbs * 1e9)) * 1e3
+
+
 def alu_floor_ms(M, N, K, levels, rank, mode, blk):
     """fp32 scales only: CUDA-core time of the per-block promotion acc += P * (sA * sB) that the chosen algorithm
     needs (the tensor core cannot apply a per-row x per-column fp32 factor per K block): M*N*(K/blk) elements,
@@ -169,6 +177,8 @@ def roofline_fractions(M, N, K, levels, rank, mode, blk, ms, pk):
     spec = combined_roofline_ms(M, N, K, levels, rank, mode, blk, SPEC_FP8_TFLOPS, SPEC_HBM_GBS)
     return {"combined_roofline_ms": meas, "combined_frac": meas / ms,
             "combined_roofline_spec_ms": spec, "combined_frac_spec": spec / ms,
+            "overlap_bound_ms": overlap_bound_ms(M, N, K, levels, rank, mode, blk, 2.0 * pk["bf16_tflops"], pk["hbm_gbs"]),
+            "overlap_bound_spec_ms": overlap_bound_ms(M, N, K, levels, rank, mode, blk, SPEC_FP8_TFLOPS, SPEC_HBM_GBS),
             "alu_floor_ms": alu_floor_ms(M, N, K, levels, rank, mode, blk)}
 
 

@@ -72,6 +72,9 @@ def test_combined_roofline_time_follows_the_derivation():
     pk = {"bf16_tflops": 1646.8, "hbm_gbs": 6459.0}
     fr = bench.roofline_fractions(n, n, n, 1, 7, "fp32", 32, 2.0385, pk)
     assert fr["combined_frac"] == pytest.approx(0.245, abs=2e-3) and fr["combined_frac_spec"] == pytest.approx(0.187, abs=2e-3)
+    # fully overlapped phases: max(tensor time, HBM time) = 213.8 us at the nominal peaks, 292.1 us at the measured ones
+    assert fr["overlap_bound_spec_ms"] == pytest.approx(0.2138, rel=2e-3)
+    assert fr["overlap_bound_ms"] == pytest.approx(0.2921, rel=2e-3)
 
 
 def test_reference_arm_prints_one_json_line():
