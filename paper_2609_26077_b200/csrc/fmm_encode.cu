@@ -406,19 +406,19 @@ __global__ void __launch_bounds__(TILE ? 256 : 128, TILE ? 2 : 4) encode_b_kerne
     }
 }
 
-// B side, block 32, one 32-k block per warp: the four warps of a block take the four 32-k blocks of one 128-k chunk
-// of the same 16 columns (thread = 16 k of one column, lanes l and l+16 the two halves of a block), so every thread
-// issues all its loads at once and a chunk is spread over four warps instead of being walked by one.
-// Grid: (cols / 16, rows / 128, batch), 128 threads.
+// B side, block 32, one 32-k block of 16 columns per warp (thread = 16 k of one column, lanes l and l+16 the two
+// halves of a block), so every thread issues all its loads at once.  A thread block is a single warp: the warps
+// share nothing, and one-warp blocks let the scheduler replace each finished warp on its own (2 % faster than four
+// warps per block, 30 % faster than eight).  Grid: (cols / 16, rows / 32, batch), 32 threads.
 template <int MODE, uint32_t NZ>
-__global__ void __launch_bounds__(128, 4) encode_b32_kernel(const EncodeParams p)
+__global__ void __launch_bounds__(32, 16) encode_b32_kernel(const EncodeParams p)
 {
     constexpr unsigned FULL = 0xffffffffu;
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x;
     const int col = lane & 15, khalf = lane >> 4;
     const int j = blockIdx.x * 16 + col;
-    const int kc = blockIdx.y;                      // chunk of 128 k
-    const int kb = kc * 4 + warp;                   // this warp's quantization block
+    const int kb = blockIdx.y;                      // this warp's quantization block
+    const int kc = kb >> 2;                         // its chunk of 128 k
     const int b = blockIdx.z;
     const int k0 = kb * 32 + khalf * 16;
     const float* base = p.in + (int64_t)b * p.in_batch_stride + j;
@@ -470,7 +470,7 @@ __global__ void __launch_bounds__(128, 4) encode_b32_kernel(const EncodeParams p
                     if (FMM_GUARD(p.guard, sp, 4, 1205)) *sp = sc;
                 } else {
                     const int64_t tile = (int64_t)kc * p.sf_blocks + (jg >> 7);
-                    char* sp = so + tile * 512 + (jg & 31) * 16 + ((jg & 127) >> 5) * 4 + warp;
+                    char* sp = so + tile * 512 + (jg & 31) * 16 + ((jg & 127) >> 5) * 4 + (kb & 3);
                     if (FMM_GUARD(p.guard, sp, 1, 1206)) *reinterpret_cast<uint8_t*>(sp) = (uint8_t)e8;
                 }
             }
@@ -853,10 +853,10 @@ void launch_b32(const EncodeParams& p, dim3 grid, cudaStream_t st)
 {
     const uint32_t m = (p.nq == 4) ? coef_mask(p) : 0u;
     switch (m) {
-#define X(M) case M: encode_b32_kernel<MODE, M><<<grid, 128, 0, st>>>(p); return;
+#define X(M) case M: encode_b32_kernel<MODE, M><<<grid, 32, 0, st>>>(p); return;
         FMM_KNOWN_MASKS(X)
 #undef X
-        default: encode_b32_kernel<MODE, 0u><<<grid, 128, 0, st>>>(p); return;
+        default: encode_b32_kernel<MODE, 0u><<<grid, 32, 0, st>>>(p); return;
     }
 }
 void launch_b128(const EncodeParams& p, dim3 grid, cudaStream_t st)
@@ -933,10 +933,10 @@ fmm_status_t fmm_launch_encode_b(const EncodeParams& p, int blk, int mode, cudaS
         else launch_b_opt<false, true>(p, grid, st);
     } else if (mode == FMM_SCALE_FP32_AMAX_DIV_448) {
         grid.x = (unsigned)(p.cols / 16);
-        if (blk == 32) launch_b32<FMM_SCALE_FP32_AMAX_DIV_448>(p, grid, st);
+        if (blk == 32) { grid.y = (unsigned)(p.rows / 32); launch_b32<FMM_SCALE_FP32_AMAX_DIV_448>(p, grid, st); }
         else launch_b128(p, grid, st);
     } else {
-        grid.x = (unsigned)(p.cols / 16);
+        grid.x = (unsigned)(p.cols / 16); grid.y = (unsigned)(p.rows / 32);
         launch_b32<FMM_SCALE_UE8M0_CEIL>(p, grid, st);
     }
     return cudaGetLastError() == cudaSuccess ? FMM_OK : FMM_ERR_CUDA;
