@@ -62,8 +62,8 @@ struct Cfg {
     static constexpr int BROWS = BN / NCTA;                  // T_r rows this CTA loads per stage
     static constexpr int A_BYTES = BM * BK;
     static constexpr int B_BYTES = BROWS * BK;
-    // The UE8M0 pair kernel is bound by operand-load latency under L2 contention: it trades epilogue
-    // staging space for more pipeline stages.
+    // The UE8M0 pair kernel keeps one staging chunk per epilogue warp: its shared memory goes to the operand stages,
+    // and a second chunk in flight per warp was measured slower (more output traffic competing with the loads).
     static constexpr int STAGING_BUFS = (MX && NCTA == 2) ? 1 : 2;
     static constexpr bool DUMP = (MODE == MODE_FP32_OUT_WARP);
     // FP32 scales per column: the promoting warps read the accumulators with the 16-lane load shape, four rows x
@@ -71,12 +71,14 @@ struct Cfg {
     // save and is faster with one row per thread.
     static constexpr bool ROWS4 = !MX && MODE != MODE_FP32_SB_TILE;
     static_assert(!DUMP || (BN == 128 && BK / BLK == 4), "output-warp mode: 128-column tiles, block 32");
-    static constexpr int STAGES = (MX && NCTA == 2) ? 6 : ((A_BYTES + B_BYTES) > 40000 || DUMP ? 3 : 4);
+    static constexpr int STAGES = (MX && NCTA == 2) ? 5 : ((A_BYTES + B_BYTES) > 40000 || DUMP ? 3 : 4);
     // DUMP (output-warp mode): shared-memory copy of a finished product, BM x BN fp32
     static constexpr int DUMP_BYTES = DUMP ? BM * BN * 4 : 0;
-    // output chunk of one epilogue warp: 32 rows x CH fp32, staged in shared memory for one TMA store
-    // (the UE8M0 pair kernel halves it: with one narrow buffer per warp a sixth operand stage fits)
-    static constexpr int CH = (MX && NCTA == 2) ? 16 : 32;
+    // output chunk of one epilogue warp: 32 rows x CH fp32, staged in shared memory for one TMA store.  Rows of 128
+    // bytes everywhere: a TMA add-reduction of 64-byte rows runs at half the bytes per clock (11 against 21 per SM,
+    // measured; plain stores 25 either way), which costs the UE8M0 pair kernel more than its sixth operand stage,
+    // bought with 16-column chunks, gave (two levels at n = 8192: 0.579 -> 0.556 ms; one level 0.451 -> 0.447 ms).
+    static constexpr int CH = 32;
     static constexpr int STAGING_BYTES = 32 * CH * 4;
     static constexpr int SFB_ATOMS = BN / 128;
     static constexpr int SF_STAGE_BYTES = MX ? (512 + SFB_ATOMS * 512) : 0;
