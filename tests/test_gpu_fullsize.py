@@ -7,25 +7,27 @@ import pytest
 import torch
 
 from oracle import oracle as O
-from paper_2609_26077_b200 import workloads as Wl
+from paper_2609_26077_b200 import fmm, workloads as Wl
 from gpu_common import MODES, coeffs, dev, make_plan
 
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("mode,blk", [("fp32", 32), ("ue8m0", 32), ("fp32", 128)])
-def test_full_size_operands_bit_exact_and_sampled_rows_of_c(mode, blk):
+@pytest.mark.parametrize("mode,blk,tile", [("fp32", 32, 0), ("ue8m0", 32, 0), ("fp32", 128, 0), ("fp32", 128, 128)])
+def test_full_size_operands_bit_exact_and_sampled_rows_of_c(mode, blk, tile):
+    # tile = 128: one weight-side scale per 128 x 128 tile (App. E.5), the fourth product-kernel mode bench.py times
     n = 8192
     h = n // 2
     A, B = Wl.gaussian(n, n, n, seed=0)
-    plan = make_plan("phi_optimal", 1, blk, mode)
+    plan = make_plan("phi_optimal", 1, blk, mode) if not tile else \
+        fmm.Plan(*coeffs("phi_optimal"), levels=1, block_k=blk, scale_mode=mode, b_tile_n=tile)
     ws = plan.workspace(n, n, n)
     C = plan.matmul(dev(A), dev(B), workspace=ws)
     torch.cuda.synchronize()
     assert plan.device_status() == (0, 0)
     U, V, W = coeffs("phi_optimal")
     ca, sa, ea = O.encode(A, "A", U, V, 1, blk, MODES[mode])
-    cb, sb, eb = O.encode(B, "B", U, V, 1, blk, MODES[mode])
+    cb, sb, eb = O.encode(B, "B", U, V, 1, blk, MODES[mode], b_tile=tile)
     rng = np.random.default_rng(1)
     rows = np.sort(rng.choice(h, size=24, replace=False))
     # four 128 x 128 tiles of the leaf index space (each is compared in all four output blocks), not aligned to the

@@ -30,12 +30,12 @@ CASES = [
     ("phi_optimal", 1, (1024, 1024, 1024), 32, "ue8m0", "gaussian"),
     ("phi_optimal", 1, (1024, 1024, 1024), 32, "fp32", "gaussian"),
     ("phi_optimal", 1, (1024, 1024, 1024), 128, "fp32", "gaussian"),
-    # more tile positions than CTA pairs / CTAs on a 148-SM part, with a short last wave: the product
-    # kernel cuts the last positions into half-width items (80 positions on 74 pairs; 152 on 148 CTAs)
     # orbit-panel arms: dense irrational coefficient tables (no compile-time zero pattern applies)
     ("pert_f1_shear_m_rb", 1, (512, 512, 512), 32, "fp32", "gaussian"),
     ("pert_f2_diag_p_rb", 1, (512, 512, 512), 32, "ue8m0", "uniform"),
     ("winograd_rb", 2, (512, 512, 512), 32, "ue8m0", "gaussian"),
+    # more tile positions than CTA pairs / CTAs on a 148-SM part (80 positions on 74 pairs; 152 on 148 CTAs): several
+    # work items per CTA (pair), spread evenly over the waves
     ("strassen", 1, (5120, 512, 4096), 32, "ue8m0", "gaussian"),
     ("phi_optimal", 1, (4864, 256, 4096), 32, "ue8m0", "uniform"),
     ("strassen", 1, (5120, 512, 4096), 128, "fp32", "gaussian"),

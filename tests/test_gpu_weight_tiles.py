@@ -17,7 +17,7 @@ CASES = [
     ("phi_optimal", 1, (512, 512, 768), "llm", True),
     ("winograd", 2, (512, 1024, 1024), "student_t3", True),
     ("pert_f0_diag_p_rb", 1, (256, 256, 512), "uniform", True),
-    # 80 tile positions on 74 CTA pairs: the last six are cut into half-width items
+    # 80 tile positions on 74 CTA pairs: two waves of 40 pairs
     ("strassen", 1, (5120, 512, 4096), "llm", False),
 ]
 
