@@ -409,7 +409,8 @@ __global__ void __launch_bounds__(TILE ? 256 : 128, TILE ? 2 : 4) encode_b_kerne
 // B side, block 32, one 32-k block of 16 columns per warp (thread = 16 k of one column, lanes l and l+16 the two
 // halves of a block), so every thread issues all its loads at once.  A thread block is a single warp: the warps
 // share nothing, and one-warp blocks let the scheduler replace each finished warp on its own (2 % faster than four
-// warps per block, 30 % faster than eight).  Grid: (cols / 16, rows / 32, batch), 32 threads.
+// warps of one 128-k chunk per block; blocks of two to eight warps side by side, covering 128- to 512-byte row
+// segments, are within 1 %).  Grid: (cols / 16, rows / 32, batch), 32 threads.
 template <int MODE, uint32_t NZ>
 __global__ void __launch_bounds__(32, 16) encode_b32_kernel(const EncodeParams p)
 {
