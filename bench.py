@@ -363,7 +363,7 @@ def run_ours(args):
             seen.add((name, lv, blk, mode))
             p2 = make_plan(name, lv, blk, mode)
             w2 = p2.workspace(M, N, K)
-            ms = time_steps(lambda: p2.matmul(A, B, out=C, workspace=w2), 5, 3)
+            ms = time_steps(lambda: p2.matmul(A, B, out=C, workspace=w2), 10, 5)
             v = {"realization": name, "levels": lv, "block_k": blk, "scale_mode": mode,
                  "ms_per_step": ms, "value": flop_eff / (ms * 1e-3) / 1e12}
             v.update(roofline_fractions(M, N, K, lv, p2.rank if lv > 0 else 8, mode, blk, ms, pk))
@@ -388,7 +388,7 @@ def run_ours(args):
                                         ("phi_optimal", 1, 32, "ue8m0"), ("strassen", 1, 32, "ue8m0"), ("cubic", 0, 32, "ue8m0")]:
                 p2 = make_plan(name, lv, blk, mode)
                 w2 = p2.workspace(Mr, Nr, Kr)
-                ms = time_steps(lambda: p2.matmul(Ar, Br, out=Cr, workspace=w2), 5, 3)
+                ms = time_steps(lambda: p2.matmul(Ar, Br, out=Cr, workspace=w2), 10, 5)
                 v = {"realization": name, "levels": lv, "block_k": blk, "scale_mode": mode, "ms_per_step": ms,
                      "value": 2.0 * Mr * Nr * Kr / (ms * 1e-3) / 1e12}
                 v.update(roofline_fractions(Mr, Nr, Kr, lv, p2.rank if lv > 0 else 8, mode, blk, ms, pk))
