@@ -131,6 +131,7 @@ fmm_status_t encode_side(const fmm_plan* plan, const FmmLayout& L, char* ws, con
         // matrix would put them.
         const bool panels = b_side ? (cols % (e.b_tile ? 512 : 256) == 0) : (rows % 4 == 0);
         e.in = X; e.in_batch_stride = 0; e.ld = cols; e.batch = 1;
+        e.overlap_prev = b_side ? 1 : 0;
         if (panels) {
             e.nq = 4; e.R = 4;
             for (int r = 0; r < 4; ++r) e.coef[r][r] = 1.0f;
@@ -173,6 +174,9 @@ fmm_status_t encode_side(const fmm_plan* plan, const FmmLayout& L, char* ws, con
             batch *= R;
         }
         e.in = cur; e.in_batch_stride = cur_stride; e.ld = cur_ld; e.batch = batch;
+        // the B-side leaf encoder may start under the tail of the A-side one (launched just before it by fmm_matmul /
+        // fmm_encode_only) when it reads the caller's matrix itself, i.e. nothing a kernel of this call has written
+        e.overlap_prev = (b_side && cur == X) ? 1 : 0;
         const int div = fused2 ? 4 : 2;
         e.rows = (int)(cur_rows / div); e.cols = (int)(cur_cols / div); e.nq = 4; e.R = R;
         e.qoff[0] = 0; e.qoff[1] = e.cols; e.qoff[2] = (int64_t)e.rows * e.ld; e.qoff[3] = (int64_t)e.rows * e.ld + e.cols;

@@ -11,6 +11,7 @@
 // Both kernels are HBM-bound streaming kernels: every input element is read once with
 // full-line coalesced loads and every output byte is written once in whole 32-byte sectors.
 #include <cuda_bf16.h>
+#include <string.h>
 #include "fmm_internal.h"
 #include "fmm_ptx.cuh"
 
@@ -205,6 +206,7 @@ __device__ __forceinline__ void store_chunk_a(const EncodeParams& p, const float
 template <int BLK, int MODE, uint32_t NZ>
 __global__ void __launch_bounds__(256) encode_a_kernel(const EncodeParams p)
 {
+    fmmptx::griddep_launch_dependents();           // the B-side encoder of the same call reads nothing written here
     constexpr int GROUP = BLK / 4;                 // lanes per block
     constexpr unsigned FULL = 0xffffffffu;
     const int lane = threadIdx.x & 31;
@@ -404,6 +406,9 @@ __global__ void __launch_bounds__(TILE ? 256 : 128, TILE ? 2 : 4) encode_b_kerne
             }
         }
     }
+    // a launch that overlapped the A-side encoder must not end before it (what follows on the stream needs both):
+    // the last block of the grid waits for it, the others leave as they finish
+    if (blockIdx.x + 1 == gridDim.x && blockIdx.y + 1 == gridDim.y && blockIdx.z + 1 == gridDim.z) fmmptx::griddep_wait();
 }
 
 // B side, block 32, one 32-k block of 16 columns per warp (thread = 16 k of one column, lanes l and l+16 the two
@@ -484,6 +489,9 @@ __global__ void __launch_bounds__(32, 16) encode_b32_kernel(const EncodeParams p
             if (FMM_GUARD(p.guard, qp, 16, 1207)) *reinterpret_cast<uint4*>(qp) = make_uint4(wv[0], wv[1], wv[2], wv[3]);
         }
     }
+    // a launch that overlapped the A-side encoder must not end before it (what follows on the stream needs both):
+    // the last block of the grid waits for it, the others leave as they finish
+    if (blockIdx.x + 1 == gridDim.x && blockIdx.y + 1 == gridDim.y && blockIdx.z + 1 == gridDim.z) fmmptx::griddep_wait();
 }
 
 // B side, block 128, per-column scales, one pass.  The four warps of a block take the four 32-k sub-blocks of one
@@ -567,6 +575,9 @@ __global__ void __launch_bounds__(128, 4) encode_b128_kernel(const EncodeParams 
             if (FMM_GUARD(p.guard, qp, 16, 1204)) *reinterpret_cast<uint4*>(qp) = make_uint4(wv[0], wv[1], wv[2], wv[3]);
         }
     }
+    // a launch that overlapped the A-side encoder must not end before it (what follows on the stream needs both):
+    // the last block of the grid waits for it, the others leave as they finish
+    if (blockIdx.x + 1 == gridDim.x && blockIdx.y + 1 == gridDim.y && blockIdx.z + 1 == gridDim.z) fmmptx::griddep_wait();
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -580,6 +591,7 @@ __global__ void __launch_bounds__(128, 4) encode_b128_kernel(const EncodeParams 
 template <int BLK, int MODE, uint32_t NZ>
 __global__ void __launch_bounds__(256) encode2_a_kernel(const EncodeParams p)
 {
+    fmmptx::griddep_launch_dependents();           // as encode_a_kernel
     constexpr int GROUP = BLK / 4;
     const int lane = threadIdx.x & 31;
     const uint32_t warp_gid = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
@@ -691,6 +703,9 @@ __global__ void __launch_bounds__(256) encode2_b_kernel(const EncodeParams p)
             }
         }
     }
+    // a launch that overlapped the A-side encoder must not end before it (what follows on the stream needs both):
+    // the last block of the grid waits for it, the others leave as they finish
+    if (blockIdx.x + 1 == gridDim.x && blockIdx.y + 1 == gridDim.y && blockIdx.z + 1 == gridDim.z) fmmptx::griddep_wait();
 }
 
 // fp32 combinations of the outer recursion levels (levels >= 3): out[b*R + r] = sum_j coef[r][j] X_j
@@ -827,6 +842,22 @@ uint32_t coef_mask(const EncodeParams& p)
 // Phi-optimal realization, and the identity used to quantize a matrix as four panels
 #define FMM_KNOWN_MASKS(X) X(0x0a5381c9u) X(0x0c385a19u) X(0x05dc8f21u) X(0x0ab3f841u) X(0x0f5fc5c9u) X(0x0cfc5f59u) X(0x00008421u)
 
+// Launch of a B-side encoder.  With p.overlap_prev it carries the programmatic-serialization attribute: the kernel
+// before it on the stream (the A-side encoder, which signals at its start) need not have drained when this one
+// begins, so its blocks fill the SMs that the other's last wave leaves idle (6 % of the encode phase at n = 8192).
+template <typename K>
+void launch_b_kernel(K kernel, dim3 grid, unsigned threads, cudaStream_t st, const EncodeParams& p)
+{
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = grid; cfg.blockDim = dim3(threads, 1, 1); cfg.stream = st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at; cfg.numAttrs = p.overlap_prev ? 1 : 0;
+    cudaLaunchKernelEx(&cfg, kernel, p);
+}
+
 template <int BLK, int MODE>
 void launch_a(const EncodeParams& p, unsigned g, cudaStream_t st)
 {
@@ -843,10 +874,10 @@ void launch_b(const EncodeParams& p, dim3 grid, cudaStream_t st)
 {
     const uint32_t m = (p.nq == 4) ? coef_mask(p) : 0u;
     switch (m) {
-#define X(M) case M: encode_b_kernel<BLK, MODE, M, false, false><<<grid, 128, 0, st>>>(p); return;
+#define X(M) case M: launch_b_kernel(encode_b_kernel<BLK, MODE, M, false, false>, grid, 128, st, p); return;
         FMM_KNOWN_MASKS(X)
 #undef X
-        default: encode_b_kernel<BLK, MODE, 0u, false, false><<<grid, 128, 0, st>>>(p); return;
+        default: launch_b_kernel(encode_b_kernel<BLK, MODE, 0u, false, false>, grid, 128, st, p); return;
     }
 }
 template <int MODE>
@@ -854,20 +885,20 @@ void launch_b32(const EncodeParams& p, dim3 grid, cudaStream_t st)
 {
     const uint32_t m = (p.nq == 4) ? coef_mask(p) : 0u;
     switch (m) {
-#define X(M) case M: encode_b32_kernel<MODE, M><<<grid, 32, 0, st>>>(p); return;
+#define X(M) case M: launch_b_kernel(encode_b32_kernel<MODE, M>, grid, 32, st, p); return;
         FMM_KNOWN_MASKS(X)
 #undef X
-        default: encode_b32_kernel<MODE, 0u><<<grid, 32, 0, st>>>(p); return;
+        default: launch_b_kernel(encode_b32_kernel<MODE, 0u>, grid, 32, st, p); return;
     }
 }
 void launch_b128(const EncodeParams& p, dim3 grid, cudaStream_t st)
 {
     const uint32_t m = (p.nq == 4) ? coef_mask(p) : 0u;
     switch (m) {
-#define X(M) case M: encode_b128_kernel<M><<<grid, 128, 0, st>>>(p); return;
+#define X(M) case M: launch_b_kernel(encode_b128_kernel<M>, grid, 128, st, p); return;
         FMM_KNOWN_MASKS(X)
 #undef X
-        default: encode_b128_kernel<0u><<<grid, 128, 0, st>>>(p); return;
+        default: launch_b_kernel(encode_b128_kernel<0u>, grid, 128, st, p); return;
     }
 }
 template <int BLK, int MODE>
@@ -884,10 +915,10 @@ template <int MODE>
 void launch_b2(const EncodeParams& p, dim3 grid, cudaStream_t st)
 {
     switch (coef_mask(p)) {
-#define X(M) case M: encode2_b_kernel<MODE, M><<<grid, 256, 0, st>>>(p); return;
+#define X(M) case M: launch_b_kernel(encode2_b_kernel<MODE, M>, grid, 256, st, p); return;
         FMM_KNOWN_MASKS(X)
 #undef X
-        default: encode2_b_kernel<MODE, 0u><<<grid, 256, 0, st>>>(p); return;
+        default: launch_b_kernel(encode2_b_kernel<MODE, 0u>, grid, 256, st, p); return;
     }
 }
 // weight-side options (tile scales and / or bf16 pre-round): blk 128, fp32 scales
@@ -898,10 +929,10 @@ void launch_b_opt(const EncodeParams& p, dim3 grid, cudaStream_t st)
     constexpr int T = TILE ? 256 : 128;
     const uint32_t m = (p.nq == 4) ? coef_mask(p) : 0u;
     switch (m) {
-#define X(M) case M: encode_b_kernel<128, F, M, TILE, PRE><<<grid, T, 0, st>>>(p); return;
+#define X(M) case M: launch_b_kernel(encode_b_kernel<128, F, M, TILE, PRE>, grid, T, st, p); return;
         FMM_KNOWN_MASKS(X)
 #undef X
-        default: encode_b_kernel<128, F, 0u, TILE, PRE><<<grid, T, 0, st>>>(p); return;
+        default: launch_b_kernel(encode_b_kernel<128, F, 0u, TILE, PRE>, grid, T, st, p); return;
     }
 }
 }  // namespace

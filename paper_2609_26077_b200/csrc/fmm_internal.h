@@ -113,6 +113,8 @@ struct EncodeParams {
     int b_tile;               // B side: 128 = one fp32 scale per 128 x 128 tile (blk 128 only), 0 = per column
     int preround_bf16;        // B side: round each combination to bfloat16 before the maximum and the cast
     FmmGuard guard;           // codes and scales of this side
+    int overlap_prev;         // B side: the kernel launched just before on the stream is the A-side encoder of the same
+                              // call (nothing this kernel reads): it may start while that one drains
 };
 
 struct CombParams {

@@ -27,6 +27,13 @@ __device__ __forceinline__ bool elect_one()
     return r != 0;
 }
 
+// Programmatic dependent launch.  launch_dependents: the next kernel on the stream, if it was launched with the
+// programmatic-serialization attribute, may start once every block of this grid has got here (or exited) instead of
+// after the grid has drained.  wait: returns when the grids this one depends on have completed and their writes are
+// visible (at once if there is no such dependency).
+__device__ __forceinline__ void griddep_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
 { asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count)); }
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
