@@ -195,10 +195,11 @@ fmm_status_t encode_side(const fmm_plan* plan, const FmmLayout& L, char* ws, con
 }
 
 fmm_status_t multiply(const fmm_plan* plan, const FmmLayout& L, char* ws, float* C, int64_t M, int64_t N,
-                      cudaStream_t st, int* launches)
+                      cudaStream_t st, int* launches, bool after_encode)
 {
     GemmParams g;
     memset(&g, 0, sizeof(g));
+    g.overlap_prev = after_encode ? 1 : 0;
     g.qa = reinterpret_cast<const uint8_t*>(ws + L.qa);
     g.qb = reinterpret_cast<const uint8_t*>(ws + L.qb);
     g.sa = ws + L.sa; g.sb = ws + L.sb;
@@ -506,7 +507,7 @@ fmm_status_t fmm_multiply_only(const fmm_plan_t* plan, float* C, int64_t M, int6
     fmm_status_t s = check_ws(plan, M, N, K, ws, ws_bytes, &L);
     if (s != FMM_OK) return s;
     int launches = 0;
-    s = multiply(plan, L, static_cast<char*>(ws), C, M, N, reinterpret_cast<cudaStream_t>(stream), &launches);
+    s = multiply(plan, L, static_cast<char*>(ws), C, M, N, reinterpret_cast<cudaStream_t>(stream), &launches, false);
     plan->last_launches.store(launches, std::memory_order_relaxed);
     return s;
 }
@@ -522,7 +523,7 @@ fmm_status_t fmm_matmul(const fmm_plan_t* plan, const float* A, const float* B, 
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
     s = encode_side(plan, L, static_cast<char*>(ws), A, M, K, false, st, &launches);
     if (s == FMM_OK) s = encode_side(plan, L, static_cast<char*>(ws), B, K, N, true, st, &launches);
-    if (s == FMM_OK) s = multiply(plan, L, static_cast<char*>(ws), C, M, N, st, &launches);
+    if (s == FMM_OK) s = multiply(plan, L, static_cast<char*>(ws), C, M, N, st, &launches, true);
     plan->last_launches.store(launches, std::memory_order_relaxed);
     return s;
 }

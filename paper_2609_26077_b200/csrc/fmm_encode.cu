@@ -406,6 +406,10 @@ __global__ void __launch_bounds__(TILE ? 256 : 128, TILE ? 2 : 4) encode_b_kerne
             }
         }
     }
+    // the product kernel, launched behind this one by the same call, may be scheduled as soon as every block has got
+    // here: its launch latency and set-up then fall under this grid's last blocks (signalling at the start instead lets
+    // its CTAs take SMs from this grid's tail: 0.5 % slower back to back)
+    fmmptx::griddep_launch_dependents();
     // a launch that overlapped the A-side encoder must not end before it (what follows on the stream needs both):
     // the last block of the grid waits for it, the others leave as they finish
     if (blockIdx.x + 1 == gridDim.x && blockIdx.y + 1 == gridDim.y && blockIdx.z + 1 == gridDim.z) fmmptx::griddep_wait();
@@ -489,6 +493,10 @@ __global__ void __launch_bounds__(32, 16) encode_b32_kernel(const EncodeParams p
             if (FMM_GUARD(p.guard, qp, 16, 1207)) *reinterpret_cast<uint4*>(qp) = make_uint4(wv[0], wv[1], wv[2], wv[3]);
         }
     }
+    // the product kernel, launched behind this one by the same call, may be scheduled as soon as every block has got
+    // here: its launch latency and set-up then fall under this grid's last blocks (signalling at the start instead lets
+    // its CTAs take SMs from this grid's tail: 0.5 % slower back to back)
+    fmmptx::griddep_launch_dependents();
     // a launch that overlapped the A-side encoder must not end before it (what follows on the stream needs both):
     // the last block of the grid waits for it, the others leave as they finish
     if (blockIdx.x + 1 == gridDim.x && blockIdx.y + 1 == gridDim.y && blockIdx.z + 1 == gridDim.z) fmmptx::griddep_wait();
@@ -575,6 +583,10 @@ __global__ void __launch_bounds__(128, 4) encode_b128_kernel(const EncodeParams 
             if (FMM_GUARD(p.guard, qp, 16, 1204)) *reinterpret_cast<uint4*>(qp) = make_uint4(wv[0], wv[1], wv[2], wv[3]);
         }
     }
+    // the product kernel, launched behind this one by the same call, may be scheduled as soon as every block has got
+    // here: its launch latency and set-up then fall under this grid's last blocks (signalling at the start instead lets
+    // its CTAs take SMs from this grid's tail: 0.5 % slower back to back)
+    fmmptx::griddep_launch_dependents();
     // a launch that overlapped the A-side encoder must not end before it (what follows on the stream needs both):
     // the last block of the grid waits for it, the others leave as they finish
     if (blockIdx.x + 1 == gridDim.x && blockIdx.y + 1 == gridDim.y && blockIdx.z + 1 == gridDim.z) fmmptx::griddep_wait();
@@ -703,6 +715,10 @@ __global__ void __launch_bounds__(256) encode2_b_kernel(const EncodeParams p)
             }
         }
     }
+    // the product kernel, launched behind this one by the same call, may be scheduled as soon as every block has got
+    // here: its launch latency and set-up then fall under this grid's last blocks (signalling at the start instead lets
+    // its CTAs take SMs from this grid's tail: 0.5 % slower back to back)
+    fmmptx::griddep_launch_dependents();
     // a launch that overlapped the A-side encoder must not end before it (what follows on the stream needs both):
     // the last block of the grid waits for it, the others leave as they finish
     if (blockIdx.x + 1 == gridDim.x && blockIdx.y + 1 == gridDim.y && blockIdx.z + 1 == gridDim.z) fmmptx::griddep_wait();

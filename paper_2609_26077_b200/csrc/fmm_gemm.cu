@@ -251,6 +251,7 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         // ------------------------------------------------------------------ TMA producer
         // (all lanes walk the loops, one elected lane issues: see the note on warp-collective issue in fmm_ptx.cuh)
         {
+            griddep_wait();        // the encoders' output is complete and visible (no-op unless launched to overlap them)
             int stage = 0; uint32_t phase = 0;
             bool ok = true;
             for (int w = unit; w < p.items && ok; w += units) {
@@ -286,6 +287,7 @@ fmm_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         // (its own thread and ring: the operand producer above has no registers to spare, and the scale ring is
         // released by the promoting warps, not by the tensor pipe)
         if (!C::MX) {
+            griddep_wait();        // as the operand producer
             int ss = 0; uint32_t sphase = 0;
             bool ok = true;
             for (int w = unit; w < p.items && ok; w += units) {
@@ -892,10 +894,14 @@ fmm_status_t launch(const GemmParams& g, cudaStream_t st)
     cfg.blockDim = dim3(NUM_THREADS, 1, 1);
     cfg.dynamicSmemBytes = C::SMEM_BYTES;
     cfg.stream = st;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = NCTA; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr; cfg.numAttrs = 1;
+    // right behind the encoders of the same call: the CTAs may be set up (barriers, TMEM, tensor maps) while the B-side
+    // encoder drains; the two producer warps wait for it before their first load
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = g.overlap_prev ? 2 : 1;
     cudaError_t ce = cudaLaunchKernelEx(&cfg, fmm_gemm_kernel<BN, MODE, BLK, NCTA>, tmA, tmB, tmC, tmSFA, tmSFB, kp);
     if (ce != cudaSuccess) { cudaGetLastError(); return FMM_ERR_CUDA; }
     return FMM_OK;

@@ -156,6 +156,8 @@ struct GemmParams {
     int* status;
     int terms_per_group;                    // consecutive terms that feed the same output blocks (R at levels >= 2, else all)
     int sb_tile;                            // fp32 scales, blk 128: the B-side scale is constant over each 128-column tile
+    int overlap_prev;                       // the kernel launched just before on the stream is the B-side encoder of the same call:
+                                            // the product kernel may be set up while that one drains (its loads wait for it)
     FmmGuard guard;                         // the output matrix (C, or the stack of parent matrices)
 };
 // guard word of the statistics kernels, which have no plan (FMM_DEBUG build; always 0 otherwise)
