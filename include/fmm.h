@@ -109,7 +109,11 @@ fmm_status_t fmm_workspace_bytes(const fmm_plan_t* plan, int64_t M, int64_t N, i
  *   The plan's device (the one current at fmm_plan_create) must be the current device: FMM_ERR_WRONG_DEVICE otherwise;
  *   the same holds for every call that takes a plan and touches the device.
  * Asynchronous on cuda_stream.  Calls sharing a workspace must be stream-ordered; a plan may be shared by host
- * threads (it is read-only during a call, apart from the launch counter below). */
+ * threads (it is read-only during a call, apart from the launch counter below).  Towards other work on the stream a
+ * call is ordinary stream-ordered work: its first kernel starts after everything enqueued before it has completed, and
+ * whatever is enqueued after it starts after all of its kernels have completed.  Between themselves the kernels of one
+ * call overlap where they do not depend on each other (programmatic dependent launch: the B-side encoder starts under
+ * the A-side encoder's last wave, the product kernel is set up under the B-side encoder's last blocks). */
 fmm_status_t fmm_matmul(const fmm_plan_t* plan, const float* A, const float* B, float* C,
                         int64_t M, int64_t N, int64_t K, void* workspace, size_t workspace_bytes,
                         void* cuda_stream);
