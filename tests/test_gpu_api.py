@@ -204,3 +204,38 @@ def test_call_on_another_device_is_refused():
     finally:
         torch.cuda.set_device(0)
     plan.close()
+
+
+@pytest.mark.parametrize("mode,blk,levels", [("fp32", 32, 1), ("ue8m0", 32, 1), ("fp32", 128, 1), ("ue8m0", 32, 2), ("fp32", 32, 0)])
+def test_work_enqueued_behind_a_call_sees_all_of_its_kernels_complete(mode, blk, levels):
+    # The kernels of one call overlap each other (the B-side encoder starts under the A-side encoder's tail, the
+    # product kernel is set up under the B side's); towards the rest of the stream the call must stay ordinary
+    # stream-ordered work.  Device-to-device copies of the workspace and of C enqueued right behind a call, with no
+    # synchronisation in between, must hold the finished bytes: they are compared with a second plan's synchronised run.
+    M, K, N = 2048, 4096, 2048
+    A, B = Wl.gaussian(M, K, N, seed=5)
+    a, b = dev(A), dev(B)
+    name = "phi_optimal" if levels else "cubic"
+    plan, ref_plan = make_plan(name, levels, blk, mode), make_plan(name, levels, blk, mode)
+    ws, ws_ref = plan.workspace(M, N, K), ref_plan.workspace(M, N, K)
+    ws_ref.zero_()
+    ref_plan.encode_only(a, b, workspace=ws_ref)
+    torch.cuda.synchronize()
+    want_encoded = ws_ref.clone()
+    want_c = ref_plan.matmul(a, b, workspace=ws_ref)
+    torch.cuda.synchronize()
+    want_after = ws_ref.clone()
+    s = torch.cuda.Stream()
+    with torch.cuda.stream(s):
+        for rep in range(4):
+            ws.zero_()
+            plan.encode_only(a, b, workspace=ws, stream=s)
+            snap_encoded = ws.clone()                         # enqueued behind the call on the same stream
+            c = torch.full((M, N), float("nan"), device="cuda")
+            plan.matmul(a, b, out=c, workspace=ws, stream=s)
+            snap_c, snap_after = c.clone(), ws.clone()
+    s.synchronize()
+    assert plan.device_status() == (0, 0)
+    assert torch.equal(snap_encoded, want_encoded), "workspace copied right behind fmm_encode_only"
+    assert torch.equal(snap_after, want_after), "workspace copied right behind fmm_matmul"
+    assert torch.equal(snap_c, want_c), "C copied right behind fmm_matmul"
